@@ -1,0 +1,158 @@
+"""Pure-Python cross-checks for the CPU checker (test-only).
+
+* ``philox_py``: Philox4x32-10 written from its published definition with Python integers.
+* ``sample_py``: the inverse-CDF rule as a literal linear scan.
+* ``brute_force``: an event-free, bookkeeping-free evaluator of the model for tiny inputs: every
+  request is a record with a status; the queue order is *derived* (waiting requests sorted by arrival
+  id), the active order is derived (sorted by activation sequence number), and every quantity is
+  recomputed from the records each slot.  It deliberately shares no structure with the C++ checker.
+"""
+from __future__ import annotations
+
+M32 = 0xFFFFFFFF
+
+
+def philox_py(ctr, key):
+    c = [int(x) & M32 for x in ctr]
+    k0, k1 = int(key[0]) & M32, int(key[1]) & M32
+    for r in range(10):
+        p0 = 0xD2511F53 * c[0]
+        p1 = 0xCD9E8D57 * c[2]
+        c = [((p1 >> 32) ^ c[1] ^ k0) & M32, p1 & M32, ((p0 >> 32) ^ c[3] ^ k1) & M32, p0 & M32]
+        k0 = (k0 + 0x9E3779B9) & M32
+        k1 = (k1 + 0xBB67AE85) & M32
+    return tuple(c)
+
+
+def sample_py(tab, u):
+    cdf = [int(x) for x in tab.cdf]
+    for k in range(len(cdf) - 1):
+        if u < cdf[k]:
+            return tab.vmin + k
+    return tab.vmin + len(cdf) - 1
+
+
+def brute_force(cfg, replica, n_steps):
+    """Returns dict(U=[..], Q=[..], completions=[(t, lat)..], counters={...}) for one replica."""
+    # locate the group
+    first = 0
+    for g in cfg.groups:
+        if replica < first + g.n_replicas:
+            grp, rid = g, g.rng_replica_base + (replica - first)
+            break
+        first += g.n_replicas
+    key = (cfg.seed & M32, (cfg.seed >> 32) & M32)
+    arr = cfg.arrivals[grp.arrivals_id]
+    reqs = []           # dicts: id, l, o, t_arr, status in {'wait','active','done'}, act_seq, p, j
+    act_seq = 0
+    state = 0
+    U_tr, Q_tr, comps = [], [], []
+    cnt = dict(arrived=0, dropped=0, admitted=0, completed=0, evictions=0, overflow_steps=0,
+               gate_blocked_steps=0, budget_blocked_steps=0, acap_blocked_steps=0, tokens_generated=0,
+               prefill_tokens=0, completed_tokens=0, wasted_tokens=0, sum_lat=0, max_lat=0, sum_U=0,
+               max_U=0, sum_N=0, max_Q=0, sum_w_completed=0)
+
+    def waiting():
+        return sorted((r for r in reqs if r["status"] == "wait"), key=lambda r: r["id"])
+
+    def active():
+        return sorted((r for r in reqs if r["status"] == "active"), key=lambda r: r["act_seq"])
+
+    def prospective():
+        # usage at the end of this slot if nothing else changes: p + j + one new token if prefilled
+        return sum(r["p"] + r["j"] + (1 if r["p"] == r["l"] else 0) for r in active())
+
+    for t in range(1, n_steps + 1):
+        w = philox_py((t, rid, 0, 0), key)
+        if arr.n_states == 2 and w[2] < arr.switch_thr[state]:
+            state ^= 1
+        n_t = sample_py(arr.count[state], w[0])
+        B_t = (grp.b_fp >> 16) + (1 if (w[1] >> 16) < (grp.b_fp & 0xFFFF) else 0)
+        for i in range(n_t):
+            a = philox_py((t, rid, 1, i), key)
+            cls = sample_py(cfg.class_law, a[0])
+            l = sample_py(cfg.prompt[cls], a[1])
+            o = sample_py(cfg.decode[cls], a[2])
+            cnt["arrived"] += 1
+            if len(waiting()) >= cfg.Qcap:
+                cnt["dropped"] += 1
+            else:
+                reqs.append(dict(id=len(reqs), l=l, o=o, t_arr=t, status="wait", act_seq=None, p=0, j=0))
+        n_dec_start = sum(1 for r in active() if r["p"] == r["l"])
+        room = None if cfg.K == 0 else (max(0, cfg.K - n_dec_start) if grp.policy == 2 else cfg.K)
+        if grp.policy == 2:
+            for r in active():
+                if r["p"] < r["l"]:
+                    g = min(grp.chunk, r["l"] - r["p"]) if room is None else min(grp.chunk, r["l"] - r["p"], room)
+                    r["p"] += g
+                    if room is not None:
+                        room -= g
+                    cnt["prefill_tokens"] += g
+        admitted_now = 0
+        while True:
+            if grp.policy == 0 and admitted_now >= B_t:
+                break
+            wq = waiting()
+            if not wq:
+                break
+            if len(active()) == cfg.Acap:
+                cnt["acap_blocked_steps"] += 1
+                break
+            h = wq[0]
+            if grp.policy == 2:
+                g = min(grp.chunk, h["l"]) if room is None else min(grp.chunk, h["l"], room)
+                if g == 0:
+                    cnt["budget_blocked_steps"] += 1
+                    break
+                need = g + (1 if g == h["l"] else 0)
+            else:
+                g = h["l"]
+                if not (room is None or admitted_now == 0 or g <= room):
+                    cnt["budget_blocked_steps"] += 1
+                    break
+                need = g + 1
+            if prospective() + need > cfg.M:
+                cnt["gate_blocked_steps"] += 1
+                break
+            h["status"], h["p"], h["j"], h["act_seq"] = "active", g, 0, act_seq
+            act_seq += 1
+            if room is not None:
+                room -= min(g, room)
+            admitted_now += 1
+            cnt["admitted"] += 1
+            cnt["prefill_tokens"] += g
+        if prospective() > cfg.M:
+            cnt["overflow_steps"] += 1
+            while prospective() > cfg.M:
+                r = active()[-1]
+                cnt["wasted_tokens"] += r["j"]
+                cnt["evictions"] += 1
+                r["status"], r["p"], r["j"], r["act_seq"] = "wait", 0, 0, None
+        for r in active():
+            if r["p"] == r["l"]:
+                r["j"] += 1
+                cnt["tokens_generated"] += 1
+        U = sum(r["p"] + r["j"] for r in active())
+        assert U <= cfg.M
+        cnt["sum_U"] += U
+        cnt["max_U"] = max(cnt["max_U"], U)
+        cnt["sum_N"] += len(active()) + len(waiting())
+        for r in active():
+            if r["p"] == r["l"] and r["j"] == r["o"]:
+                lat = t - r["t_arr"] + 1
+                r["status"] = "done"
+                comps.append((t, lat))
+                cnt["completed"] += 1
+                cnt["sum_lat"] += lat
+                cnt["max_lat"] = max(cnt["max_lat"], lat)
+                cnt["completed_tokens"] += r["o"]
+                cnt["sum_w_completed"] += sum(r["l"] + jj for jj in range(1, r["o"] + 1))
+        U_tr.append(U)
+        Q_tr.append(len(waiting()))
+        cnt["max_Q"] = max(cnt["max_Q"], len(waiting()))
+    cnt["q_final"] = len(waiting())
+    cnt["p_final"] = len(active())
+    cnt["resid_age"] = sum(n_steps - r["t_arr"] + 1 for r in reqs if r["status"] in ("wait", "active"))
+    cnt["resid_j"] = sum(r["j"] for r in active())
+    cnt["mmpp_state"] = state
+    return dict(U=U_tr, Q=Q_tr, completions=comps, counters=cnt)
