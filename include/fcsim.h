@@ -1,0 +1,196 @@
+/*
+ * fcsim -- batched Monte-Carlo evaluation of the token-level LLM-serving model on one GPU.
+ *
+ * Each replica is an independent copy of the discrete-time single-worker system of Section 2.1:
+ * requests (l, o, t_arr) arrive n_t per slot into a FIFO waiting queue, are activated into an active
+ * set whose KV-cache usage U_t = sum (l_i + j_i(t)) must stay <= M, generate one output token per
+ * slot, and leave at the end of the slot in which the last token is produced.  Activation follows
+ * Algorithm 2 (flow control: at most B_t activations per slot, E[B_t] = b, Theorem 3.6) with
+ * last-in-first-out eviction on overflow (Section 3.3), or one of two baselines named in the
+ * Introduction: greedy prefill-first admission (the b -> infinity limit of Algorithm 2) and chunked
+ * prefill.  Metrics are those of Section 2.2: token throughput, prompt throughput, latency.
+ *
+ * All simulation state and arithmetic are integers.  Random words come from Philox4x32-10 with key =
+ * seed and counter = (slot, replica id, stream, index); stream 0 (index 0) gives the slot's words
+ * (word 0 -> n_t, word 1 -> B_t, word 2 -> arrival-state switch), stream 1 (index i) gives arrival i
+ * of the slot (word 0 -> class, word 1 -> l, word 2 -> o).
+ *
+ * Conventions: every function returns 0 (FCSIM_OK) or a negative error code; nothing throws, aborts
+ * or traps.  "HOST" / "DEVICE" says where a pointer must live.  Device output buffers are allocated
+ * and owned by the caller; the library only allocates small private device copies of the tables.
+ * One GPU; a handle is bound to the device that is current in fcsim_create.
+ */
+#ifndef FCSIM_H
+#define FCSIM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    FCSIM_OK = 0,
+    FCSIM_EINVAL = -1, /* bad field, non-monotone table, vmin < 1 for a length table, max l + max o > M, ... */
+    FCSIM_ECAP = -2,   /* Qcap/Acap need more shared memory than one warp can be given */
+    FCSIM_ESIZE = -3,  /* a required buffer is NULL or too small */
+    FCSIM_ERANGE = -4, /* steps beyond T_max */
+    FCSIM_ECUDA = -5,  /* CUDA runtime error; code via fcsim_last_cuda_error */
+    FCSIM_ENOMEM = -6  /* host allocation failed */
+};
+
+enum { FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2 };
+
+/* Integer inverse-CDF table.  Support {vmin .. vmin+n-1}; cdf[k] = floor(P(X <= vmin+k) * 2^32) clamped
+ * to 2^32-1, non-decreasing; cdf[n-1] is a catch-all whose value is ignored.  A 32-bit word u maps to
+ * vmin + min{k < n-1 : u < cdf[k]}, or vmin+n-1 if there is none.  `cdf` is a HOST pointer borrowed only
+ * for the duration of fcsim_create / fcsim_query_sizes / fcsim_simulate_host. */
+typedef struct {
+    uint32_t n;
+    int32_t vmin;
+    const uint32_t* cdf;
+} fcsim_table;
+
+/* Law of the arrival count n_t (Section 2.1: n_t drawn from a known law with mean lambda).
+ * n_states = 1: one count table.  n_states = 2: two-state modulated law; each slot the state s flips
+ * first iff word 2 of the slot < switch_thr[s], then n_t is drawn from count[s].  Initial state 0.
+ * Count values must lie in [0, 255]. */
+typedef struct {
+    uint32_t n_states;
+    fcsim_table count[2];
+    uint32_t switch_thr[2];
+} fcsim_arrivals;
+
+/* A group of replicas sharing policy and parameters; replicas are laid out group after group.
+ * b_fp: Q16.16 activation rate b of Algorithm 2; B_t = (b_fp >> 16) + [ (word1 >> 16) < (b_fp & 0xffff) ],
+ *       i.i.d., mean b_fp / 65536, bounded by (b_fp >> 16) + 1 (the law asked for by Theorem 3.6).
+ * chunk: prefill chunk size c (CHUNKED only, >= 1).
+ * rng_replica_base: generator replica id of the group's first replica (equal bases in two groups give
+ *       common random numbers). */
+typedef struct {
+    int32_t policy;
+    uint32_t b_fp;
+    int32_t chunk;
+    int32_t arrivals_id;
+    uint32_t rng_replica_base;
+    int32_t n_replicas;
+} fcsim_group;
+
+/* M: KV capacity in tokens (1 .. 2^30).  K: prefill-token budget per slot, 0 = none (the paper's model).
+ * T_max: horizon (1 .. 2^24-1).  Qcap: waiting room; a new arrival finding |Q| >= Qcap is dropped and
+ * counted (evicted requests always re-enter).  Acap: storage bound of the active set; when it is full,
+ * activation stops for the slot and acap_blocked_steps counts it.  Lengths l, o must lie in [1, 65535],
+ * n_classes in [1, 256].  All table/array pointers are HOST pointers. */
+typedef struct {
+    int32_t M, K, T_max, Qcap, Acap;
+    uint64_t seed;
+    int32_t n_classes;
+    fcsim_table class_law;     /* values 0 .. n_classes-1 */
+    const fcsim_table* prompt; /* [n_classes] law of l per class */
+    const fcsim_table* decode; /* [n_classes] law of o per class */
+    int32_t n_arrivals;
+    const fcsim_arrivals* arrivals;
+    int32_t n_groups;
+    const fcsim_group* groups;
+    int32_t trace_stride; /* record {U_t, |Q_t|} when t % stride == 0; 0 = no trace */
+    int32_t hist_bins;    /* 0 = no latency histogram; bin = min(latency >> hist_shift, hist_bins-1) */
+    int32_t hist_shift;
+    int32_t complog_cap;  /* completions logged per replica; 0 = no log */
+} fcsim_config;
+
+/* Per-replica counters, all int64, accumulated over the slots run so far (R = number of replicas).
+ * Latency of a request = t_done - t_arr + 1 slots (arrival to completion, Section 2.2).
+ * sum_w_completed adds l*o + o(o+1)/2 per completion (the per-request workload of Prop. 3.2).
+ * status: bit 0 = Acap was hit, bit 1 = completion log overflowed.  q_final, p_final, resid_age
+ * (sum over unfinished requests of t - t_arr + 1), resid_j (output tokens held by active requests) and
+ * mmpp_state describe the state at the last slot run. */
+typedef struct {
+    int64_t steps_done, status, arrived, dropped, admitted, completed, evictions, overflow_steps,
+        gate_blocked_steps, budget_blocked_steps, acap_blocked_steps, tokens_generated, prefill_tokens,
+        completed_tokens, wasted_tokens, sum_lat, max_lat, sum_U, max_U, sum_N, max_Q, sum_w_completed,
+        n_logged, q_final, p_final, resid_age, resid_j, mmpp_state;
+} fcsim_counters;
+
+/* Per-group summary: `total` combines the group's replicas field by field (sum; max for max_lat, max_U,
+ * max_Q and steps_done; bitwise or for status).  With n = replicas in the group and T = slots run:
+ * mean_latency = sum_lat / completed; mean_utilisation = sum_U / (n T M); request_throughput =
+ * completed / (n T); token_throughput = tokens_generated / (n T) (Section 2.2); p95/p99: smallest
+ * histogram bin k whose cumulative count reaches ceil(q * completed / 100), reported as
+ * ((k+1) << hist_shift) - 1, or max_lat for the open last bin; 0 when there is no histogram or no
+ * completion. */
+typedef struct {
+    fcsim_counters total;
+    double mean_latency, p95_latency, p99_latency, mean_utilisation, request_throughput, token_throughput;
+} fcsim_summary;
+
+/* DEVICE buffers, caller-owned, each at least the size fcsim_query_sizes reports and 16-byte aligned.
+ * workspace: per-replica simulator state between launches (scratch; opaque).
+ * counters:  [R] fcsim_counters.
+ * trace:     [R][T_max / trace_stride] {int32 U_t, int32 |Q_t|}, or NULL when trace_stride = 0.
+ * hist:      [R][hist_bins] int32, or NULL when hist_bins = 0.
+ * complog:   [R][complog_cap] {int32 t_done, int32 latency}, or NULL when complog_cap = 0.
+ * scratch:   per-group reduction area used by fcsim_stats (opaque). */
+typedef struct {
+    void* workspace;
+    void* counters;
+    void* trace;
+    void* hist;
+    void* complog;
+    void* scratch;
+} fcsim_buffers;
+
+typedef struct {
+    size_t workspace, counters, trace, hist, complog, scratch;
+} fcsim_sizes;
+
+/* Launch geometry chosen for a handle (for reporting). */
+typedef struct {
+    int32_t grid, block, warps_per_block, blocks_per_sm, sm_count;
+    int32_t smem_per_block, smem_per_warp, max_steps_per_launch;
+} fcsim_launch_info;
+
+typedef struct fcsim fcsim_t; /* opaque host object */
+
+/* Validates `cfg` and reports the bytes the caller must allocate for each device buffer. */
+int fcsim_query_sizes(const fcsim_config* cfg, fcsim_sizes* out);
+
+/* Validates, copies the tables to the device, zeroes workspace/counters/hist/complog/trace and returns a
+ * handle positioned before slot 1.  Synchronous (default stream).  The buffers must outlive the handle. */
+int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* device_buffers, fcsim_t** out);
+
+/* Advances every replica by n_steps slots (steps_done + n_steps <= T_max, else FCSIM_ERANGE).
+ * Asynchronous on `cuda_stream` (a cudaStream_t; NULL = default stream).  Resumable: run(a) then run(b)
+ * gives bit for bit the state and outputs of run(a+b).  Long runs are split into several launches. */
+int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream);
+
+/* Reduces counters and histograms per group on the device, then synchronises `cuda_stream` and copies:
+ * host_out (HOST, [R], may be NULL) <- per-replica counters; per_group_out (HOST, [n_groups], may be
+ * NULL) <- summaries. */
+int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_out, fcsim_summary* per_group_out);
+
+int fcsim_destroy(fcsim_t* h);
+
+int32_t fcsim_steps_done(const fcsim_t* h);
+int fcsim_get_launch_info(const fcsim_t* h, fcsim_launch_info* out);
+int fcsim_last_cuda_error(const fcsim_t* h); /* cudaError_t of the last FCSIM_ECUDA, else 0 */
+const char* fcsim_last_cuda_error_name(const fcsim_t* h); /* its symbolic name */
+
+/* Diagnostics.  A library compiled with -DFCSIM_CHECKED compares every shared-memory and output index of
+ * the step kernel with its bound; the first violation is recorded instead of performed.  fcsim_debug_read
+ * copies the record to HOST out[8] = {source line (0 = none), index, bound, replica, 0, 0, 0, 0}
+ * (synchronous).  In a normal build the record is always zero. */
+int fcsim_debug_read(fcsim_t* h, uint32_t out[8]);
+int fcsim_is_checked_build(void);
+const char* fcsim_strerror(int code);
+
+/* Whole job with HOST buffers: allocates device buffers (cudaMalloc), runs slots 1..n_steps, copies the
+ * outputs to the given HOST arrays (each may be NULL; shapes as in fcsim_buffers with T_max = cfg->T_max)
+ * and frees the device memory.  Synchronous. */
+int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcsim_counters* host_counters,
+                        void* host_trace, void* host_hist, void* host_complog, fcsim_summary* per_group_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FCSIM_H */

@@ -1,0 +1,547 @@
+// Host side of fcsim: validation, table upload, launch geometry, resumable runs, statistics.
+// The C ABI is declared in include/fcsim.h.
+#include "fcsim.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "fcsim_device.cuh"
+
+using namespace fcsim_dev;
+
+static_assert(sizeof(fcsim_counters) == C_COUNT * sizeof(int64_t), "counter block layout");
+
+namespace {
+
+constexpr size_t kSmemBudget = 227 * 1024;   // shared memory one CTA may opt in to
+constexpr int kMaxStepsPerLaunch = 32768;    // keeps the 32-bit per-launch partial sums exact
+constexpr long long kTargetWorkPerLaunch = 1LL << 31;  // replica-steps per launch (bounds launch time)
+constexpr int kStatsChunk = 256;             // replicas reduced by one block before it touches the group row
+
+struct Layout {
+    int RC, Apad, S;
+    size_t ws_stride, smem_per_warp;
+    int warps_per_block;
+    int n_rec;
+    long long R;
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool table_ok(const fcsim_table& t, int64_t vmin_lo, int64_t vmax_hi) {
+    if (t.n == 0 || t.cdf == nullptr) return false;
+    if (t.vmin < vmin_lo || (int64_t)t.vmin + (int64_t)t.n - 1 > vmax_hi) return false;
+    for (uint32_t k = 1; k + 1 < t.n; ++k)
+        if (t.cdf[k] < t.cdf[k - 1]) return false;
+    return true;
+}
+
+// Validates the description and derives the storage layout.  Returns an FCSIM_* code.
+int plan(const fcsim_config* c, Layout* L) {
+    if (!c) return FCSIM_EINVAL;
+    if (c->M < 1 || c->M > (1 << 30) || c->K < 0 || c->T_max < 1 || c->T_max >= (1 << 24)) return FCSIM_EINVAL;
+    if (c->Qcap < 1 || c->Acap < 1) return FCSIM_EINVAL;
+    if (c->n_classes < 1 || c->n_classes > 256 || !c->prompt || !c->decode) return FCSIM_EINVAL;
+    if (c->n_arrivals < 1 || !c->arrivals || c->n_groups < 1 || !c->groups) return FCSIM_EINVAL;
+    if (!table_ok(c->class_law, 0, c->n_classes - 1) || c->class_law.vmin != 0 ||
+        (int)c->class_law.n != c->n_classes)
+        return FCSIM_EINVAL;
+    int64_t lmax = 0, omax = 0;
+    for (int k = 0; k < c->n_classes; ++k) {
+        if (!table_ok(c->prompt[k], 1, 65535) || !table_ok(c->decode[k], 1, 65535)) return FCSIM_EINVAL;
+        lmax = std::max<int64_t>(lmax, (int64_t)c->prompt[k].vmin + c->prompt[k].n - 1);
+        omax = std::max<int64_t>(omax, (int64_t)c->decode[k].vmin + c->decode[k].n - 1);
+    }
+    if (lmax + omax > c->M) return FCSIM_EINVAL;  // a single request must fit the cache
+    int max_count = 0;
+    for (int a = 0; a < c->n_arrivals; ++a) {
+        const fcsim_arrivals& A = c->arrivals[a];
+        if (A.n_states != 1 && A.n_states != 2) return FCSIM_EINVAL;
+        for (uint32_t s = 0; s < A.n_states; ++s) {
+            if (!table_ok(A.count[s], 0, 255)) return FCSIM_EINVAL;
+            max_count = std::max<int>(max_count, A.count[s].vmin + (int)A.count[s].n - 1);
+        }
+    }
+    long long R = 0;
+    for (int g = 0; g < c->n_groups; ++g) {
+        const fcsim_group& G = c->groups[g];
+        if (G.policy < 0 || G.policy > 2 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.arrivals_id < 0 || G.arrivals_id >= c->n_arrivals) return FCSIM_EINVAL;
+        if (G.policy == FCSIM_POLICY_CHUNKED && G.chunk < 1) return FCSIM_EINVAL;
+        R += G.n_replicas;
+    }
+    if (R > 0x7fffffffLL) return FCSIM_EINVAL;
+    if (c->trace_stride < 0 || c->hist_bins < 0 || c->hist_shift < 0 || c->hist_shift > 30 || c->complog_cap < 0)
+        return FCSIM_EINVAL;
+
+    const long long rc = (long long)c->Qcap + c->Acap;  // evictions may push the queue past Qcap
+    if (rc > (1 << 20)) return FCSIM_ECAP;
+    L->RC = (int)align_up((size_t)rc, 2);
+    L->Apad = (int)align_up((size_t)c->Acap, 4);
+    L->S = (int)align_up((size_t)std::max(64, max_count), 2);
+    L->ws_stride = kHeaderWords * 4 + (size_t)L->RC * 8 + (size_t)L->Apad * 4;
+    L->smem_per_warp = (size_t)L->RC * 8 + (size_t)L->Apad * 4 + (size_t)L->S * 8;
+    if (L->smem_per_warp > kSmemBudget) return FCSIM_ECAP;
+    int w = kWarpsPerBlock;
+    while (w > 1 && (size_t)w * L->smem_per_warp > kSmemBudget) w >>= 1;
+    L->warps_per_block = w;
+    L->n_rec = c->trace_stride > 0 ? c->T_max / c->trace_stride : 0;
+    L->R = R;
+    return FCSIM_OK;
+}
+
+void sizes_of(const fcsim_config* c, const Layout& L, fcsim_sizes* s) {
+    s->workspace = (size_t)L.R * L.ws_stride;
+    s->counters = (size_t)L.R * sizeof(fcsim_counters);
+    s->trace = (size_t)L.R * (size_t)L.n_rec * 8;
+    s->hist = (size_t)L.R * (size_t)c->hist_bins * 4;
+    s->complog = (size_t)L.R * (size_t)c->complog_cap * 8;
+    s->scratch = (size_t)c->n_groups * ((size_t)C_COUNT + (size_t)c->hist_bins) * 8;
+}
+
+// ---- statistics kernels ---------------------------------------------------------------------------
+// Group rows in scratch: [n_groups][C_COUNT] int64 counters, then [n_groups][hist_bins] int64 bins.
+
+__device__ __forceinline__ int group_of(const DevGroup* groups, int n_groups, int r) {
+    int lo = 0, hi = n_groups - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (groups[mid].first <= r) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ void combine_into(long long* dst, int field, long long v) {
+    if (field == C_MAX_LAT || field == C_MAX_U || field == C_MAX_Q || field == C_STEPS_DONE)
+        atomicMax(dst, v);
+    else if (field == C_STATUS)
+        atomicOr(reinterpret_cast<unsigned long long*>(dst), (unsigned long long)v);
+    else
+        atomicAdd(reinterpret_cast<unsigned long long*>(dst), (unsigned long long)v);
+}
+
+__device__ __forceinline__ long long combine(int field, long long a, long long b) {
+    if (field == C_MAX_LAT || field == C_MAX_U || field == C_MAX_Q || field == C_STEPS_DONE) return a > b ? a : b;
+    if (field == C_STATUS) return a | b;
+    return a + b;
+}
+
+// One warp per chunk of replicas; lane k owns counter field k.
+__global__ void reduce_counters_kernel(const long long* __restrict__ counters, const DevGroup* __restrict__ groups,
+                                       int n_groups, int n_replicas, int chunk, long long* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int n_warps = (gridDim.x * blockDim.x) >> 5;
+    const int n_chunks = (n_replicas + chunk - 1) / chunk;
+    for (int c = warp; c < n_chunks; c += n_warps) {
+        const int r0 = c * chunk, r1 = min(n_replicas, r0 + chunk);
+        int g = group_of(groups, n_groups, r0);
+        int g_end = groups[g].first + groups[g].n;
+        long long acc = 0;
+        for (int r = r0; r < r1; ++r) {
+            if (r >= g_end) {
+                if (lane < C_COUNT) combine_into(out + (size_t)g * C_COUNT + lane, lane, acc);
+                acc = 0;
+                ++g;
+                g_end = groups[g].first + groups[g].n;
+            }
+            if (lane < C_COUNT) acc = combine(lane, acc, counters[(size_t)r * C_COUNT + lane]);
+        }
+        if (lane < C_COUNT) combine_into(out + (size_t)g * C_COUNT + lane, lane, acc);
+    }
+}
+
+// One block per chunk of replicas; thread b walks bins b, b+blockDim, .. (coalesced rows).
+__global__ void reduce_hist_kernel(const int* __restrict__ hist, const DevGroup* __restrict__ groups, int n_groups,
+                                   int n_replicas, int bins, int chunk, long long* __restrict__ out) {
+    const int n_chunks = (n_replicas + chunk - 1) / chunk;
+    for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+        const int r0 = c * chunk, r1 = min(n_replicas, r0 + chunk);
+        for (int b = threadIdx.x; b < bins; b += blockDim.x) {
+            int g = group_of(groups, n_groups, r0);
+            int g_end = groups[g].first + groups[g].n;
+            long long acc = 0;
+            for (int r = r0; r < r1; ++r) {
+                if (r >= g_end) {
+                    if (acc) atomicAdd(reinterpret_cast<unsigned long long*>(out + (size_t)g * bins + b),
+                                       (unsigned long long)acc);
+                    acc = 0;
+                    ++g;
+                    g_end = groups[g].first + groups[g].n;
+                }
+                acc += hist[(size_t)r * bins + b];
+            }
+            if (acc) atomicAdd(reinterpret_cast<unsigned long long*>(out + (size_t)g * bins + b),
+                               (unsigned long long)acc);
+        }
+    }
+}
+
+}  // namespace
+
+struct fcsim {
+    fcsim_config cfg;                 // scalar fields only; the pointers inside are not kept
+    std::vector<fcsim_group> groups;  // host copy
+    Layout L;
+    fcsim_buffers buf;
+    Params params;
+    uint32_t* d_pool = nullptr;
+    DevTable* d_tables = nullptr;
+    DevArrivals* d_arrivals = nullptr;
+    DevGroup* d_groups = nullptr;
+    unsigned int* d_work = nullptr;
+    int device = 0, sm_count = 0, blocks_per_sm = 1, grid = 1;
+    int t_done = 0;
+    int last_cuda = 0;
+    size_t table_bytes = 0;
+};
+
+#define CUDA_TRY(h, call)                                 \
+    do {                                                  \
+        cudaError_t e__ = (call);                         \
+        if (e__ != cudaSuccess) {                         \
+            (h)->last_cuda = (int)e__;                    \
+            return FCSIM_ECUDA;                           \
+        }                                                 \
+    } while (0)
+
+extern "C" int fcsim_query_sizes(const fcsim_config* cfg, fcsim_sizes* out) {
+    if (!out) return FCSIM_EINVAL;
+    Layout L;
+    const int rc = plan(cfg, &L);
+    if (rc != FCSIM_OK) return rc;
+    sizes_of(cfg, L, out);
+    return FCSIM_OK;
+}
+
+static int upload_tables(fcsim* h, const fcsim_config* c) {
+    std::vector<uint32_t> pool;
+    auto add = [&](const fcsim_table& t) {
+        DevTable d;
+        d.off = (uint32_t)pool.size();
+        d.n = t.n;
+        d.vmin = t.vmin;
+        d.pad = 0;
+        pool.insert(pool.end(), t.cdf, t.cdf + t.n);
+        return d;
+    };
+    std::vector<DevTable> tables;
+    tables.push_back(add(c->class_law));
+    for (int k = 0; k < c->n_classes; ++k) tables.push_back(add(c->prompt[k]));
+    for (int k = 0; k < c->n_classes; ++k) tables.push_back(add(c->decode[k]));
+    std::vector<DevArrivals> arrs(c->n_arrivals);
+    for (int a = 0; a < c->n_arrivals; ++a) {
+        const fcsim_arrivals& A = c->arrivals[a];
+        arrs[a].n_states = A.n_states;
+        arrs[a].pad = 0;
+        arrs[a].count[0] = add(A.count[0]);
+        arrs[a].count[1] = A.n_states == 2 ? add(A.count[1]) : arrs[a].count[0];
+        arrs[a].thr[0] = A.switch_thr[0];
+        arrs[a].thr[1] = A.switch_thr[1];
+    }
+    std::vector<DevGroup> grps(c->n_groups);
+    int first = 0;
+    for (int g = 0; g < c->n_groups; ++g) {
+        const fcsim_group& G = c->groups[g];
+        grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas, 0};
+        first += G.n_replicas;
+    }
+    CUDA_TRY(h, cudaMalloc(&h->d_pool, pool.size() * sizeof(uint32_t)));
+    CUDA_TRY(h, cudaMalloc(&h->d_tables, tables.size() * sizeof(DevTable)));
+    CUDA_TRY(h, cudaMalloc(&h->d_arrivals, arrs.size() * sizeof(DevArrivals)));
+    CUDA_TRY(h, cudaMalloc(&h->d_groups, grps.size() * sizeof(DevGroup)));
+    CUDA_TRY(h, cudaMalloc(&h->d_work, 16 * sizeof(unsigned int)));
+    CUDA_TRY(h, cudaMemset(h->d_work, 0, 16 * sizeof(unsigned int)));
+    CUDA_TRY(h, cudaMemcpy(h->d_pool, pool.data(), pool.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    CUDA_TRY(h, cudaMemcpy(h->d_tables, tables.data(), tables.size() * sizeof(DevTable), cudaMemcpyHostToDevice));
+    CUDA_TRY(h, cudaMemcpy(h->d_arrivals, arrs.data(), arrs.size() * sizeof(DevArrivals), cudaMemcpyHostToDevice));
+    CUDA_TRY(h, cudaMemcpy(h->d_groups, grps.data(), grps.size() * sizeof(DevGroup), cudaMemcpyHostToDevice));
+    h->table_bytes = pool.size() * 4 + tables.size() * sizeof(DevTable) + arrs.size() * sizeof(DevArrivals) +
+                     grps.size() * sizeof(DevGroup);
+    return FCSIM_OK;
+}
+
+static void release(fcsim* h) {
+    if (!h) return;
+    cudaFree(h->d_pool);
+    cudaFree(h->d_tables);
+    cudaFree(h->d_arrivals);
+    cudaFree(h->d_groups);
+    cudaFree(h->d_work);
+    delete h;
+}
+
+extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_t** out) {
+    if (!out) return FCSIM_EINVAL;
+    *out = nullptr;
+    Layout L;
+    int rc = plan(cfg, &L);
+    if (rc != FCSIM_OK) return rc;
+    if (!b) return FCSIM_ESIZE;
+    fcsim_sizes sz;
+    sizes_of(cfg, L, &sz);
+    if (!b->workspace || !b->counters || !b->scratch) return FCSIM_ESIZE;
+    if (sz.trace && !b->trace) return FCSIM_ESIZE;
+    if (sz.hist && !b->hist) return FCSIM_ESIZE;
+    if (sz.complog && !b->complog) return FCSIM_ESIZE;
+    const void* ptrs[6] = {b->workspace, b->counters, b->trace, b->hist, b->complog, b->scratch};
+    for (const void* q : ptrs)
+        if (q && (reinterpret_cast<uintptr_t>(q) & 15)) return FCSIM_ESIZE;
+
+    fcsim* h = new (std::nothrow) fcsim();
+    if (!h) return FCSIM_ENOMEM;
+    h->cfg = *cfg;
+    h->cfg.prompt = h->cfg.decode = nullptr;
+    h->cfg.arrivals = nullptr;
+    h->cfg.class_law.cdf = nullptr;
+    h->groups.assign(cfg->groups, cfg->groups + cfg->n_groups);
+    h->cfg.groups = nullptr;
+    h->L = L;
+    h->buf = *b;
+
+    auto fail = [&](int code) {
+        const int keep = h->last_cuda;
+        release(h);
+        (void)keep;
+        return code;
+    };
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e != cudaSuccess) return fail(FCSIM_ECUDA);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, h->device);
+    if (e != cudaSuccess) return fail(FCSIM_ECUDA);
+    h->sm_count = prop.multiProcessorCount;
+    rc = upload_tables(h, cfg);
+    if (rc != FCSIM_OK) return fail(rc);
+
+    const size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
+    if (smem_block > (size_t)prop.sharedMemPerBlockOptin) return fail(FCSIM_ECAP);
+    e = cudaFuncSetAttribute(fcsim_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block);
+    if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fcsim_step_kernel, L.warps_per_block * 32, smem_block);
+    if (e != cudaSuccess || occ < 1) { h->last_cuda = (int)e; return fail(e != cudaSuccess ? FCSIM_ECUDA : FCSIM_ECAP); }
+    h->blocks_per_sm = occ;
+    const long long want = (L.R + L.warps_per_block - 1) / L.warps_per_block;
+    h->grid = (int)std::max<long long>(1, std::min<long long>((long long)h->sm_count * occ, want));
+
+    // zeroed buffers are the state "before slot 1"
+    const struct { void* p; size_t n; } z[] = {{b->workspace, sz.workspace}, {b->counters, sz.counters},
+                                               {b->trace, sz.trace},         {b->hist, sz.hist},
+                                               {b->complog, sz.complog},     {b->scratch, sz.scratch}};
+    for (const auto& it : z) {
+        if (it.p && it.n) {
+            e = cudaMemset(it.p, 0, it.n);
+            if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+        }
+    }
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+
+    Params& p = h->params;
+    std::memset(&p, 0, sizeof(p));
+    p.M = cfg->M; p.K = cfg->K; p.Qcap = cfg->Qcap; p.Acap = cfg->Acap;
+    p.RC = L.RC; p.S = L.S; p.Apad = L.Apad;
+    p.key0 = (uint32_t)(cfg->seed & 0xffffffffu);
+    p.key1 = (uint32_t)(cfg->seed >> 32);
+    p.n_classes = cfg->n_classes; p.n_groups = cfg->n_groups; p.n_replicas = (int)L.R;
+    p.trace_stride = cfg->trace_stride; p.n_rec = L.n_rec;
+    p.hist_bins = cfg->hist_bins; p.hist_shift = cfg->hist_shift; p.complog_cap = cfg->complog_cap;
+    p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
+    p.workspace = static_cast<unsigned char*>(b->workspace);
+    p.ws_stride = L.ws_stride;
+    p.counters = static_cast<long long*>(b->counters);
+    p.trace = L.n_rec > 0 ? static_cast<int2*>(b->trace) : nullptr;
+    p.hist = cfg->hist_bins > 0 ? static_cast<int*>(b->hist) : nullptr;
+    p.complog = cfg->complog_cap > 0 ? static_cast<int2*>(b->complog) : nullptr;
+    p.work_counter = h->d_work;
+    p.debug = h->d_work + 8;
+    p.smem_per_warp = (uint32_t)L.smem_per_warp;
+    *out = h;
+    return FCSIM_OK;
+}
+
+static int max_steps_per_launch(const fcsim* h) {
+    long long s = kTargetWorkPerLaunch / std::max<long long>(1, h->L.R);
+    s = std::max<long long>(256, std::min<long long>(s, kMaxStepsPerLaunch));
+    return (int)s;
+}
+
+extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
+    if (!h || n_steps < 0) return FCSIM_EINVAL;
+    if ((long long)h->t_done + n_steps > h->cfg.T_max) return FCSIM_ERANGE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int per = max_steps_per_launch(h);
+    const size_t smem_block = (size_t)h->L.warps_per_block * h->L.smem_per_warp;
+    int left = n_steps;
+    while (left > 0) {
+        const int now = std::min(left, per);
+        Params p = h->params;
+        p.t0 = h->t_done;
+        p.n_steps = now;
+        CUDA_TRY(h, cudaMemsetAsync(h->d_work, 0, sizeof(unsigned int), st));
+        fcsim_step_kernel<<<h->grid, h->L.warps_per_block * 32, smem_block, st>>>(p);
+        CUDA_TRY(h, cudaGetLastError());
+        h->t_done += now;
+        left -= now;
+    }
+    return FCSIM_OK;
+}
+
+static double percentile(const long long* hist, int bins, int shift, long long n, int q, long long max_lat) {
+    if (n <= 0 || bins <= 0) return 0.0;
+    const long long target = (q * n + 99) / 100;
+    long long cum = 0;
+    int k = 0;
+    for (; k < bins; ++k) {
+        cum += hist[k];
+        if (cum >= target) break;
+    }
+    if (k >= bins - 1) return (double)max_lat;
+    return (double)((((long long)k + 1) << shift) - 1);
+}
+
+extern "C" int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_out, fcsim_summary* per_group_out) {
+    if (!h) return FCSIM_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int G = (int)h->groups.size();
+    const int bins = h->cfg.hist_bins;
+    const int R = (int)h->L.R;
+    std::vector<long long> host_scratch;
+    if (per_group_out) {
+        long long* d_cnt = static_cast<long long*>(h->buf.scratch);
+        long long* d_hist = d_cnt + (size_t)G * C_COUNT;
+        const size_t bytes = (size_t)G * ((size_t)C_COUNT + bins) * 8;
+        CUDA_TRY(h, cudaMemsetAsync(h->buf.scratch, 0, bytes, st));
+        const int n_chunks = (R + kStatsChunk - 1) / kStatsChunk;
+        {
+            const int warps_per_block = 8;
+            const int blocks = std::max(1, std::min((n_chunks + warps_per_block - 1) / warps_per_block, h->sm_count * 8));
+            reduce_counters_kernel<<<blocks, warps_per_block * 32, 0, st>>>(
+                static_cast<const long long*>(h->buf.counters), h->d_groups, G, R, kStatsChunk, d_cnt);
+            CUDA_TRY(h, cudaGetLastError());
+        }
+        if (bins > 0) {
+            const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
+            reduce_hist_kernel<<<blocks, 256, 0, st>>>(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins,
+                                                       kStatsChunk, d_hist);
+            CUDA_TRY(h, cudaGetLastError());
+        }
+        host_scratch.resize(bytes / 8);
+        CUDA_TRY(h, cudaMemcpyAsync(host_scratch.data(), h->buf.scratch, bytes, cudaMemcpyDeviceToHost, st));
+    }
+    if (host_out)
+        CUDA_TRY(h, cudaMemcpyAsync(host_out, h->buf.counters, (size_t)R * sizeof(fcsim_counters),
+                                    cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(h, cudaStreamSynchronize(st));
+    if (per_group_out) {
+        const double T = (double)h->t_done;
+        for (int g = 0; g < G; ++g) {
+            fcsim_summary& s = per_group_out[g];
+            std::memcpy(&s.total, host_scratch.data() + (size_t)g * C_COUNT, sizeof(fcsim_counters));
+            const double n = (double)h->groups[g].n_replicas;
+            const fcsim_counters& c = s.total;
+            s.mean_latency = c.completed > 0 ? (double)c.sum_lat / (double)c.completed : 0.0;
+            s.mean_utilisation = T > 0 ? (double)c.sum_U / (n * T * (double)h->cfg.M) : 0.0;
+            s.request_throughput = T > 0 ? (double)c.completed / (n * T) : 0.0;
+            s.token_throughput = T > 0 ? (double)c.tokens_generated / (n * T) : 0.0;
+            const long long* gh = host_scratch.data() + (size_t)G * C_COUNT + (size_t)g * bins;
+            s.p95_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 95, c.max_lat);
+            s.p99_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 99, c.max_lat);
+        }
+    }
+    return FCSIM_OK;
+}
+
+extern "C" int fcsim_destroy(fcsim_t* h) {
+    if (!h) return FCSIM_EINVAL;
+    release(h);
+    return FCSIM_OK;
+}
+
+extern "C" int32_t fcsim_steps_done(const fcsim_t* h) { return h ? h->t_done : -1; }
+
+extern "C" int fcsim_get_launch_info(const fcsim_t* h, fcsim_launch_info* out) {
+    if (!h || !out) return FCSIM_EINVAL;
+    out->grid = h->grid;
+    out->block = h->L.warps_per_block * 32;
+    out->warps_per_block = h->L.warps_per_block;
+    out->blocks_per_sm = h->blocks_per_sm;
+    out->sm_count = h->sm_count;
+    out->smem_per_block = (int32_t)(h->L.warps_per_block * h->L.smem_per_warp);
+    out->smem_per_warp = (int32_t)h->L.smem_per_warp;
+    out->max_steps_per_launch = max_steps_per_launch(h);
+    return FCSIM_OK;
+}
+
+extern "C" int fcsim_last_cuda_error(const fcsim_t* h) { return h ? h->last_cuda : 0; }
+
+extern "C" const char* fcsim_last_cuda_error_name(const fcsim_t* h) {
+    return cudaGetErrorName(static_cast<cudaError_t>(h ? h->last_cuda : 0));
+}
+
+extern "C" int fcsim_debug_read(fcsim_t* h, uint32_t out[8]) {
+    if (!h || !out) return FCSIM_EINVAL;
+    CUDA_TRY(h, cudaMemcpy(out, h->d_work + 8, 8 * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return FCSIM_OK;
+}
+
+extern "C" int fcsim_is_checked_build(void) {
+#ifdef FCSIM_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+extern "C" const char* fcsim_strerror(int code) {
+    switch (code) {
+        case FCSIM_OK: return "ok";
+        case FCSIM_EINVAL: return "invalid argument or configuration";
+        case FCSIM_ECAP: return "Qcap/Acap do not fit the shared memory of one warp";
+        case FCSIM_ESIZE: return "a required buffer is missing, misaligned or too small";
+        case FCSIM_ERANGE: return "steps beyond T_max";
+        case FCSIM_ECUDA: return "CUDA runtime error";
+        case FCSIM_ENOMEM: return "host allocation failed";
+        default: return "unknown error";
+    }
+}
+
+extern "C" int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcsim_counters* host_counters,
+                                   void* host_trace, void* host_hist, void* host_complog,
+                                   fcsim_summary* per_group_out) {
+    fcsim_sizes sz;
+    int rc = fcsim_query_sizes(cfg, &sz);
+    if (rc != FCSIM_OK) return rc;
+    fcsim_buffers b;
+    std::memset(&b, 0, sizeof(b));
+    void** slots[6] = {&b.workspace, &b.counters, &b.trace, &b.hist, &b.complog, &b.scratch};
+    const size_t bytes[6] = {sz.workspace, sz.counters, sz.trace, sz.hist, sz.complog, sz.scratch};
+    auto free_all = [&]() {
+        for (void** s : slots) cudaFree(*s);
+    };
+    for (int i = 0; i < 6; ++i) {
+        if (bytes[i] && cudaMalloc(slots[i], bytes[i]) != cudaSuccess) {
+            free_all();
+            return FCSIM_ECUDA;
+        }
+    }
+    fcsim_t* h = nullptr;
+    rc = fcsim_create(cfg, &b, &h);
+    if (rc == FCSIM_OK) rc = fcsim_run(h, n_steps, nullptr);
+    if (rc == FCSIM_OK) rc = fcsim_stats(h, nullptr, host_counters, per_group_out);
+    if (rc == FCSIM_OK) {
+        cudaError_t e = cudaSuccess;
+        if (host_trace && sz.trace) e = cudaMemcpy(host_trace, b.trace, sz.trace, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && host_hist && sz.hist) e = cudaMemcpy(host_hist, b.hist, sz.hist, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && host_complog && sz.complog)
+            e = cudaMemcpy(host_complog, b.complog, sz.complog, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) rc = FCSIM_ECUDA;
+    }
+    if (h) fcsim_destroy(h);
+    free_all();
+    return rc;
+}

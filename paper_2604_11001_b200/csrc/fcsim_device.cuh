@@ -1,0 +1,585 @@
+// Device side of fcsim: one warp advances one replica of the serving model of Section 2.1
+// under Algorithm 2 (or the greedy / chunked-prefill baselines), slot by slot.
+//
+// Data layout per replica (shared memory while a warp owns the replica, the same bytes in the
+// caller's workspace between launches):
+//   ring  [RC]   u64   waiting queue and active set in ONE ring: entries head .. head+nP-1 are the
+//                      active set in activation order, the next nQ entries are the FIFO queue.
+//                      Because activation is FIFO and eviction is LIFO back to the queue front
+//                      (Section 3.3), the concatenation is always sorted by arrival, so activation
+//                      and eviction only move the boundary; nothing is copied.
+//                      entry = l | o << 16 | t_arr << 32 | class << 56.
+//   state [Acap] u32   one word per active entry (its own ring, same order): for a request whose
+//                      prompt is in the cache the slot in which its last token is generated
+//                      (t_fin = activation slot + o - 1, so its output count is implied by the
+//                      slot number and "process all requests" costs nothing); for a request still
+//                      prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so far.
+//   stage [S]    u64   arrivals generated ahead of time for the next batch of <= 32 slots.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace fcsim_dev {
+
+constexpr int kWarpsPerBlock = 4;
+constexpr int kHeaderWords = 16;  // per-replica scalar state kept in the workspace
+constexpr uint32_t kNoFin = 0xFFFFFFFFu;
+constexpr uint32_t kPrefillBit = 0x80000000u;
+
+enum CounterIdx {
+    C_STEPS_DONE = 0, C_STATUS, C_ARRIVED, C_DROPPED, C_ADMITTED, C_COMPLETED, C_EVICTIONS,
+    C_OVERFLOW_STEPS, C_GATE_BLOCKED, C_BUDGET_BLOCKED, C_ACAP_BLOCKED, C_TOKENS_GENERATED,
+    C_PREFILL_TOKENS, C_COMPLETED_TOKENS, C_WASTED_TOKENS, C_SUM_LAT, C_MAX_LAT, C_SUM_U, C_MAX_U,
+    C_SUM_N, C_MAX_Q, C_SUM_W_COMPLETED, C_N_LOGGED, C_Q_FINAL, C_P_FINAL, C_RESID_AGE, C_RESID_J,
+    C_MMPP_STATE, C_COUNT
+};
+
+struct DevTable {
+    uint32_t off;  // first threshold in the pool
+    uint32_t n;
+    int32_t vmin;
+    uint32_t pad;
+};
+struct DevArrivals {
+    DevTable count[2];
+    uint32_t thr[2];
+    uint32_t n_states;
+    uint32_t pad;
+};
+struct DevGroup {
+    int32_t policy;
+    uint32_t b_fp;
+    int32_t chunk;
+    int32_t arrivals_id;
+    uint32_t rng_base;
+    int32_t first;  // index of the group's first replica
+    int32_t n;
+    int32_t pad;
+};
+
+struct Params {
+    int32_t M, K, Qcap, Acap, RC, S, Apad;  // RC, Apad: padded storage sizes of the two rings
+    uint32_t key0, key1;
+    int32_t n_classes, n_groups, n_replicas;
+    int32_t trace_stride, n_rec, hist_bins, hist_shift, complog_cap;
+    int32_t t0, n_steps;
+    const uint32_t* pool;         // all thresholds
+    const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
+    const DevArrivals* arrivals;
+    const DevGroup* groups;
+    unsigned char* workspace;     // [R] records of ws_stride bytes
+    unsigned long long ws_stride;
+    long long* counters;          // [R][C_COUNT]
+    int2* trace;
+    int* hist;
+    int2* complog;
+    unsigned int* work_counter;
+    unsigned int* debug;          // 8 words: first failed index check (checked build), else untouched
+    uint32_t smem_per_warp;
+};
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and xors,
+// key schedule k += (0x9E3779B9, 0xBB67AE85).
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t& o0, uint32_t& o1, uint32_t& o2,
+                                              uint32_t& o3) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    o0 = c0; o1 = c1; o2 = c2; o3 = c3;
+}
+
+// vmin + (first k < n-1 with thresholds[k] > u, else n-1).
+__device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, const DevTable tb, uint32_t u) {
+    const uint32_t* __restrict__ cdf = pool + tb.off;
+    uint32_t lo = 0, hi = tb.n - 1;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(cdf + mid) > u) hi = mid; else lo = mid + 1;
+    }
+    return tb.vmin + (int)lo;
+}
+
+__device__ __forceinline__ uint32_t lanemask_gt() {
+    uint32_t m;
+    asm("mov.u32 %0, %%lanemask_gt;" : "=r"(m));
+    return m;
+}
+
+__device__ __forceinline__ int warp_incl_scan(int v, int lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+
+__device__ __forceinline__ long long warp_sum64(long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
+}
+
+__device__ __forceinline__ uint64_t pack_entry(int l, int o, int t_arr, int cls) {
+    return (uint64_t)(uint32_t)(l | (o << 16)) | ((uint64_t)(uint32_t)(t_arr | (cls << 24)) << 32);
+}
+__device__ __forceinline__ int entry_l(uint64_t e) { return (int)((uint32_t)e & 0xffffu); }
+__device__ __forceinline__ int entry_o(uint64_t e) { return (int)((uint32_t)e >> 16); }
+__device__ __forceinline__ int entry_tarr(uint64_t e) { return (int)((uint32_t)(e >> 32) & 0xffffffu); }
+
+// Index-checked build (-DFCSIM_CHECKED): every shared-memory and output index is compared with its
+// bound; a bad one is recorded (line, index, bound, replica) in Params::debug and the access goes to a
+// dummy location instead, so a logic error shows up as a report, never as a memory fault.
+#ifdef FCSIM_CHECKED
+template <typename T>
+__device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limit, int line, unsigned int* dbg,
+                                          unsigned int replica) {
+    __shared__ T dummy[kWarpsPerBlock * 32];
+    if (idx >= 0 && idx < limit) return base[idx];
+    if (atomicCAS(dbg, 0u, (unsigned)line) == 0u) {
+        dbg[1] = (unsigned)idx;
+        dbg[2] = (unsigned)limit;
+        dbg[3] = replica;
+    }
+    return dummy[threadIdx.x];
+}
+#define RING(i) checked_ref(ring, (i), RC, __LINE__, p.debug, r)
+#define STATE(i) checked_ref(state, (i), Acap, __LINE__, p.debug, r)
+#define STAGE(i) checked_ref(stage, (i), S, __LINE__, p.debug, r)
+#define TROW(i) checked_ref(trow, (i), p.n_rec, __LINE__, p.debug, r)
+#define LROW(i) checked_ref(lrow, (i), p.complog_cap, __LINE__, p.debug, r)
+#define HROW(i) checked_ref(hrow, (i), p.hist_bins, __LINE__, p.debug, r)
+#else
+#define RING(i) ring[(i)]
+#define STATE(i) state[(i)]
+#define STAGE(i) stage[(i)]
+#define TROW(i) trow[(i)]
+#define LROW(i) lrow[(i)]
+#define HROW(i) hrow[(i)]
+#endif
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const Params p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    unsigned char* my = smem_raw + (size_t)warp * p.smem_per_warp;
+    uint64_t* ring = reinterpret_cast<uint64_t*>(my);
+    uint32_t* state = reinterpret_cast<uint32_t*>(my + (size_t)p.RC * 8);
+    uint64_t* stage = reinterpret_cast<uint64_t*>(my + (size_t)p.RC * 8 + (size_t)p.Apad * 4);
+    const int state_bytes = p.RC * 8 + p.Apad * 4;  // multiple of 16 (host guarantees)
+
+    const int RC = p.RC, Acap = p.Acap, Qcap = p.Qcap, M = p.M, K = p.K, S = p.S;
+    const bool kinf = (K == 0);
+    const uint32_t FULL = 0xffffffffu;
+    const uint32_t gt_mask = lanemask_gt();
+
+    for (;;) {
+        // ------------------------------------------------------------------ next replica
+        unsigned int r = 0;
+        if (lane == 0) r = atomicAdd(p.work_counter, 1u);
+        r = __shfl_sync(FULL, r, 0);
+        if (r >= (unsigned)p.n_replicas) break;
+
+        int gi = 0;
+        {
+            int lo = 0, hi = p.n_groups - 1;
+            while (lo < hi) {  // last group whose first replica is <= r
+                const int mid = (lo + hi + 1) >> 1;
+                if (p.groups[mid].first <= (int)r) lo = mid; else hi = mid - 1;
+            }
+            gi = lo;
+        }
+        const DevGroup grp = p.groups[gi];
+        const DevArrivals arr = p.arrivals[grp.arrivals_id];
+        const uint32_t rid = grp.rng_base + (r - (unsigned)grp.first);
+        const int policy = grp.policy;
+        const int chunk = grp.chunk;
+        const bool two_state = arr.n_states == 2;
+
+        // ------------------------------------------------------------------ load state
+        unsigned char* ws = p.workspace + (size_t)r * p.ws_stride;
+        uint32_t* hdr = reinterpret_cast<uint32_t*>(ws);
+        const uint32_t hw = (lane < kHeaderWords) ? hdr[lane] : 0u;
+        int head = (int)__shfl_sync(FULL, hw, 0);
+        int shead = (int)__shfl_sync(FULL, hw, 1);
+        int nP = (int)__shfl_sync(FULL, hw, 2);
+        int nQ = (int)__shfl_sync(FULL, hw, 3);
+        int U = (int)__shfl_sync(FULL, hw, 4);        // usage carried out of the last slot, completions released
+        int Ndec = (int)__shfl_sync(FULL, hw, 5);     // active requests whose prompt is fully in the cache
+        uint32_t next_fin = ~__shfl_sync(FULL, hw, 6);  // stored complemented so that zeroed memory means "none"
+        int n_pref = (int)__shfl_sync(FULL, hw, 7);   // active requests still prefilling
+        int pf_lo = (int)__shfl_sync(FULL, hw, 8);    // lower bound on the index of the oldest of those
+        uint32_t mstate = __shfl_sync(FULL, hw, 9);
+        uint32_t status = __shfl_sync(FULL, hw, 10);
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(ws + kHeaderWords * 4);
+            uint4* dst = reinterpret_cast<uint4*>(my);
+            for (int i = lane; i < state_bytes / 16; i += 32) dst[i] = src[i];
+        }
+        long long* cptr = p.counters + (size_t)r * C_COUNT;
+        long long cnt = (lane < C_COUNT) ? cptr[lane] : 0;  // lane k owns counter k
+        __syncwarp();
+
+// The value is evaluated by every lane BEFORE the lane test: arguments may contain warp-wide primitives.
+#define CADD(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt += v__; } while (0)
+#define CMAX(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt = (cnt > v__) ? cnt : v__; } while (0)
+#define CSET(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt = v__; } while (0)
+#define WR(x) ((x) >= RC ? (x) - RC : (x))
+#define WA(x) ((x) >= Acap ? (x) - Acap : (x))
+
+        // per-launch partial sums of the quantities touched every slot
+        unsigned long long sumU = 0;
+        uint32_t sumN = 0, tokgen = 0, arrived = 0;
+        int maxU = 0, maxQ = 0;
+        int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
+
+        int t = p.t0;
+        const int t_end = p.t0 + p.n_steps;
+
+        // trace bookkeeping: lane (rec & 31) holds record rec until its block of 32 is flushed
+        const int stride = p.trace_stride;
+        int rec = stride > 0 ? t / stride : 0;
+        int cd = stride > 0 ? stride - (t % stride) : 0;
+        const int rec_lo = rec;
+        int tr_u = 0, tr_q = 0;
+        int2* trow = p.trace ? p.trace + (size_t)r * p.n_rec : nullptr;
+        int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
+        int2* lrow = p.complog ? p.complog + (size_t)r * p.complog_cap : nullptr;
+
+        while (t < t_end) {
+            // -------------------------------------------------------------- batch: draws of up to 32 slots
+            int L = min(32, t_end - t);
+            uint32_t w0, w1, w2, w3;
+            philox4x32_10((uint32_t)(t + 1 + lane), rid, 0u, 0u, p.key0, p.key1, w0, w1, w2, w3);
+            const int Bt = (int)(grp.b_fp >> 16) + (((w1 >> 16) < (grp.b_fp & 0xffffu)) ? 1 : 0);
+            int n = sample_table(p.pool, arr.count[0], w0);
+            uint32_t smask = 0;  // bit k = arrival state in slot t+1+k
+            if (two_state) {
+                const int n1 = sample_table(p.pool, arr.count[1], w0);
+                const uint32_t f0 = __ballot_sync(FULL, w2 < arr.thr[0]);
+                const uint32_t f1 = __ballot_sync(FULL, w2 < arr.thr[1]);
+                uint32_t cur = mstate;
+                for (int k = 0; k < 32; ++k) {
+                    cur ^= ((cur ? f1 : f0) >> k) & 1u;
+                    smask |= cur << k;
+                }
+                if ((smask >> lane) & 1u) n = n1;
+            }
+            if (lane >= L) n = 0;
+            int incl = warp_incl_scan(n, lane);
+            L = min(L, __popc(__ballot_sync(FULL, incl <= S)));  // staged arrivals must fit; n <= S so L >= 1
+            if (lane >= L) n = 0;
+            const int excl = incl - n;
+            const int N = __shfl_sync(FULL, incl, L - 1);
+            // generate the N arrivals of these slots, one per lane (stream 1, index = rank within the slot)
+            for (int base = 0; base < N; base += 32) {
+                const int idx = base + lane;
+                int lo = 0, hi = L - 1;
+#pragma unroll
+                for (int it = 0; it < 5; ++it) {  // slot k = first with incl_k > idx
+                    const int mid = (lo + hi) >> 1;
+                    const int v = __shfl_sync(FULL, incl, mid);
+                    if (lo < hi) { if (v > idx) hi = mid; else lo = mid + 1; }
+                }
+                const int ex_k = __shfl_sync(FULL, excl, lo);
+                if (idx < N) {
+                    uint32_t a0, a1, a2, a3;
+                    philox4x32_10((uint32_t)(t + 1 + lo), rid, 1u, (uint32_t)(idx - ex_k), p.key0, p.key1, a0, a1,
+                                  a2, a3);
+                    const int cls = sample_table(p.pool, p.tables[0], a0);
+                    const int l = sample_table(p.pool, p.tables[1 + cls], a1);
+                    const int o = sample_table(p.pool, p.tables[1 + p.n_classes + cls], a2);
+                    STAGE(idx) = pack_entry(l, o, t + 1 + lo, cls);
+                }
+            }
+            __syncwarp();
+            const uint32_t packed = (uint32_t)n | ((uint32_t)Bt << 8);
+
+            // -------------------------------------------------------------- the slots of the batch
+            for (int k = 0; k < L; ++k) {
+                ++t;
+                const uint32_t info = __shfl_sync(FULL, packed, k);
+                const int ex = __shfl_sync(FULL, excl, k);
+                const int n_t = (int)(info & 0xffu);
+                const int B_t = (int)(info >> 8);
+
+                // ---- arrivals join the queue tail; a full waiting room drops the rest
+                if (n_t > 0) {
+                    const int acc = min(n_t, max(0, Qcap - nQ));
+                    const int tail = head + nP + nQ;
+                    for (int i = lane; i < acc; i += 32) RING(WR(WR(tail) + i)) = STAGE(ex + i);
+                    nQ += acc;
+                    arrived += n_t;
+                    if (acc < n_t) CADD(C_DROPPED, n_t - acc);
+                    __syncwarp();
+                }
+
+                // ---- usage the slot would reach, token room
+                int G = U + Ndec;
+                int R = (policy == 2) ? max(0, K - Ndec) : K;
+
+                // ---- chunked policy: continuing prefills first, in activation order
+                if (policy == 2 && n_pref > 0) {
+                    int first_left = -1;
+                    for (int base = pf_lo; base < nP; base += 32) {
+                        const int i = base + lane;
+                        uint32_t sw = 0;
+                        uint64_t e = 0;
+                        if (i < nP) { sw = STATE(WA(shead + i)); e = RING(WR(head + i)); }
+                        const bool pf = (sw & kPrefillBit) != 0;
+                        const int pcur = (int)(sw & ~kPrefillBit);
+                        const int l = entry_l(e);
+                        const int d = pf ? min(chunk, l - pcur) : 0;
+                        const int dincl = warp_incl_scan(d, lane);
+                        int g = d;
+                        if (!kinf) g = min(d, max(0, R - (dincl - d)));
+                        const bool fin = pf && (pcur + g == l);
+                        if (pf && g > 0) {
+                            STATE(WA(shead + i)) = fin ? (uint32_t)(t + entry_o(e) - 1) : (kPrefillBit | (uint32_t)(pcur + g));
+                        }
+                        const int gsum = __reduce_add_sync(FULL, g);
+                        const uint32_t finm = __ballot_sync(FULL, fin);
+                        const uint32_t leftm = __ballot_sync(FULL, pf && !fin);
+                        const int nfin = __popc(finm);
+                        if (!kinf) R -= gsum;
+                        G += gsum + nfin;
+                        CADD(C_PREFILL_TOKENS, gsum);
+                        Ndec += nfin;
+                        n_pref -= nfin;
+                        if (finm) {
+                            const uint32_t mine = fin ? (uint32_t)(t + entry_o(e) - 1) : kNoFin;
+                            next_fin = min(next_fin, __reduce_min_sync(FULL, mine));
+                        }
+                        if (first_left < 0 && leftm) first_left = base + (__ffs(leftm) - 1);
+                        if (!kinf && R == 0 && first_left >= 0) break;  // nothing more can move this slot
+                    }
+                    if (first_left >= 0) pf_lo = first_left;
+                    __syncwarp();
+                }
+
+                // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
+                {
+                    int a = 0;
+                    const int cap = (policy == 0) ? B_t : 0x7fffffff;
+                    while (a < cap && nQ > 0) {
+                        if (nP == Acap) { CADD(C_ACAP_BLOCKED, 1); status |= 1u; break; }
+                        const uint64_t e = RING(WR(head + nP));
+                        const int l = entry_l(e);
+                        int g, need;
+                        if (policy == 2) {
+                            g = kinf ? min(chunk, l) : min(min(chunk, l), R);
+                            if (g == 0) { CADD(C_BUDGET_BLOCKED, 1); break; }
+                            need = g + (g == l ? 1 : 0);
+                        } else {
+                            g = l;
+                            if (!(kinf || a == 0 || g <= R)) { CADD(C_BUDGET_BLOCKED, 1); break; }
+                            need = l + 1;
+                        }
+                        if (G + need > M) { CADD(C_GATE_BLOCKED, 1); break; }
+                        uint32_t sw;
+                        if (g == l) {
+                            sw = (uint32_t)(t + entry_o(e) - 1);
+                            next_fin = min(next_fin, sw);
+                            Ndec++;
+                        } else {
+                            sw = kPrefillBit | (uint32_t)g;
+                            if (n_pref == 0) pf_lo = nP;
+                            n_pref++;
+                        }
+                        if (lane == 0) STATE(WA(shead + nP)) = sw;
+                        nP++;
+                        nQ--;
+                        G += need;
+                        if (!kinf) R -= min(g, R);
+                        a++;
+                        CADD(C_PREFILL_TOKENS, g);
+                    }
+                    if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
+                }
+
+                // ---- overflow: evict the most recently activated until the slot fits (LIFO, Section 3.3);
+                //      evicted requests lose all progress and are again the head of the queue
+                if (G > M) {
+                    CADD(C_OVERFLOW_STEPS, 1);
+                    int nev = 0, wasted = 0;
+                    while (G > M && nP > 0) {
+                        const int i = nP - 1;
+                        const uint32_t sw = STATE(WA(shead + i));
+                        if (sw & kPrefillBit) {
+                            G -= (int)(sw & ~kPrefillBit);
+                            n_pref--;
+                        } else {
+                            const uint64_t e = RING(WR(head + i));
+                            const int j = t - (int)sw + entry_o(e) - 1;  // tokens generated before this slot
+                            G -= entry_l(e) + j + 1;
+                            wasted += j;
+                            Ndec--;
+                        }
+                        nP--;
+                        nQ++;
+                        nev++;
+                    }
+                    if (pf_lo > nP) pf_lo = nP;
+                    CADD(C_EVICTIONS, nev);
+                    CADD(C_WASTED_TOKENS, wasted);
+                }
+
+                // ---- process: one token per request whose prompt is in the cache; U_t = G
+                tokgen += Ndec;
+                U = G;
+                sumU += (unsigned)G;
+                maxU = max(maxU, G);
+                sumN += nP + nQ;
+
+                // ---- retire the requests that generated their last token in this slot
+                if ((uint32_t)t == next_fin) {
+                    uint32_t newmin = kNoFin;
+                    int ndone = 0, top = -1;
+                    for (int base = 0; base < nP; base += 32) {
+                        const int i = base + lane;
+                        const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kNoFin;
+                        const bool done = (sw == (uint32_t)t);
+                        const uint32_t m = __ballot_sync(FULL, done);
+                        if (m) { ndone += __popc(m); top = base + 31 - __clz(m); }
+                        if (!done) newmin = min(newmin, sw);
+                    }
+                    next_fin = __reduce_min_sync(FULL, newmin);
+                    if (ndone > 0) {
+                        int holes = 0;  // completions at higher indices than the current block
+                        int sum_lat = 0, sum_o = 0, sum_lo = 0, max_lat = 0;
+                        long long sum_w = 0;
+                        for (int base = top & ~31; base >= 0; base -= 32) {
+                            const int i = base + lane;
+                            const bool valid = i <= top;
+                            uint32_t sw = kNoFin;
+                            uint64_t e = 0;
+                            if (valid) { sw = STATE(WA(shead + i)); e = RING(WR(head + i)); }
+                            const bool done = valid && (sw == (uint32_t)t);
+                            const uint32_t m = __ballot_sync(FULL, done);
+                            const int sh = holes + __popc(m & gt_mask);  // completions after this entry
+                            if (done) {
+                                const int l = entry_l(e), o = entry_o(e);
+                                const int lat = t - entry_tarr(e) + 1;
+                                sum_lat += lat;
+                                sum_o += o;
+                                sum_lo += l + o;
+                                max_lat = max(max_lat, lat);
+                                sum_w += (long long)l * o + (long long)o * (o + 1) / 2;
+                                if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
+                                if (lrow) {
+                                    const int li = n_logged + ndone - 1 - sh;  // log is in activation order
+                                    if (li < p.complog_cap) LROW(li) = make_int2(t, lat);
+                                }
+                            }
+                            __syncwarp();
+                            if (valid && !done && sh > 0) {  // survivors slide up over the holes
+                                RING(WR(head + i + sh)) = e;
+                                STATE(WA(shead + i + sh)) = sw;
+                            }
+                            __syncwarp();
+                            holes += __popc(m);
+                        }
+                        head = WR(head + ndone);
+                        shead = WA(shead + ndone);
+                        nP -= ndone;
+                        Ndec -= ndone;
+                        pf_lo = max(0, pf_lo - ndone);
+                        U -= __reduce_add_sync(FULL, sum_lo);
+                        CADD(C_COMPLETED, ndone);
+                        CADD(C_SUM_LAT, __reduce_add_sync(FULL, sum_lat));
+                        CADD(C_COMPLETED_TOKENS, __reduce_add_sync(FULL, sum_o));
+                        CMAX(C_MAX_LAT, __reduce_max_sync(FULL, max_lat));
+                        const long long sw_all = warp_sum64(sum_w);
+                        CADD(C_SUM_W_COMPLETED, sw_all);
+                        if (lrow) {
+                            if (n_logged + ndone > p.complog_cap) status |= 2u;
+                            n_logged = min(p.complog_cap, n_logged + ndone);
+                        }
+                    }
+                }
+
+                // ---- record
+                maxQ = max(maxQ, nQ);
+                if (stride > 0 && --cd == 0) {
+                    cd = stride;
+                    if (lane == (rec & 31)) { tr_u = G; tr_q = nQ; }
+                    if ((rec & 31) == 31) {
+                        const int b0 = rec & ~31;
+                        if (b0 + lane >= rec_lo) TROW(b0 + lane) = make_int2(tr_u, tr_q);
+                    }
+                    rec++;
+                }
+            }  // slots of the batch
+            if (two_state) mstate = (smask >> (L - 1)) & 1u;
+        }  // while t < t_end
+
+        // ------------------------------------------------------------------ flush, final extras, spill
+        if (stride > 0 && (rec & 31) != 0) {
+            const int b0 = rec & ~31;
+            if (b0 + lane >= rec_lo && b0 + lane < rec) TROW(b0 + lane) = make_int2(tr_u, tr_q);
+        }
+        long long age = 0, resj = 0;
+        for (int i = lane; i < nP + nQ; i += 32) {
+            const uint64_t e = RING(WR(head + i));
+            age += t_end - entry_tarr(e) + 1;
+            if (i < nP) {
+                const uint32_t sw = STATE(WA(shead + i));
+                if (!(sw & kPrefillBit)) resj += t_end - (int)sw + entry_o(e);
+            }
+        }
+        age = warp_sum64(age);
+        resj = warp_sum64(resj);
+        CADD(C_SUM_U, sumU);
+        CADD(C_SUM_N, sumN);
+        CADD(C_TOKENS_GENERATED, tokgen);
+        CADD(C_ARRIVED, arrived);
+        CMAX(C_MAX_U, maxU);
+        CMAX(C_MAX_Q, maxQ);
+        CSET(C_STEPS_DONE, t_end);
+        CSET(C_STATUS, status);
+        CSET(C_N_LOGGED, n_logged);
+        CSET(C_Q_FINAL, nQ);
+        CSET(C_P_FINAL, nP);
+        CSET(C_RESID_AGE, age);
+        CSET(C_RESID_J, resj);
+        CSET(C_MMPP_STATE, mstate);
+        if (lane < C_COUNT) cptr[lane] = cnt;
+
+        uint32_t out = 0;
+        switch (lane) {
+            case 0: out = (uint32_t)head; break;
+            case 1: out = (uint32_t)shead; break;
+            case 2: out = (uint32_t)nP; break;
+            case 3: out = (uint32_t)nQ; break;
+            case 4: out = (uint32_t)U; break;
+            case 5: out = (uint32_t)Ndec; break;
+            case 6: out = ~next_fin; break;
+            case 7: out = (uint32_t)n_pref; break;
+            case 8: out = (uint32_t)pf_lo; break;
+            case 9: out = mstate; break;
+            case 10: out = status; break;
+            default: break;
+        }
+        if (lane < kHeaderWords) hdr[lane] = out;
+        {
+            uint4* dst = reinterpret_cast<uint4*>(ws + kHeaderWords * 4);
+            const uint4* src = reinterpret_cast<const uint4*>(my);
+            for (int i = lane; i < state_bytes / 16; i += 32) dst[i] = src[i];
+        }
+        __syncwarp();
+#undef CADD
+#undef CMAX
+#undef CSET
+#undef WR
+#undef WA
+    }
+}
+
+}  // namespace fcsim_dev

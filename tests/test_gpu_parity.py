@@ -1,0 +1,123 @@
+"""GPU parity: the CUDA library against the CPU checker, word for word, through the C ABI."""
+import os
+
+import numpy as np
+import pytest
+
+from gpu_common import assert_same, assert_summary_close, run_gpu
+from helpers import degenerate_config, read_fixture, scaled_presets, trace_fixtures
+from oracle import fcsim_oracle as orc
+from paper_2604_11001_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+@pytest.mark.parametrize("name", trace_fixtures(GOLDEN))
+def test_hand_traces_on_gpu(name):
+    fx = read_fixture(os.path.join(GOLDEN, name))
+    cfg = degenerate_config(**fx["params"])
+    gpu = run_gpu(cfg)
+    assert gpu["trace"][0, :, 0].tolist() == fx["U"]
+    assert gpu["trace"][0, :, 1].tolist() == fx["Q"]
+    n = int(gpu["counters"][0, orc.CIDX["n_logged"]])
+    assert [tuple(x) for x in gpu["complog"][0, :n].tolist()] == fx["completions"]
+    assert_same(cfg, gpu, orc.run(cfg), cfg.T_max, name)
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_random_small_configs(seed):
+    cfg = wl.random_small_config(seed, n_replicas=5, T=97)
+    gpu = run_gpu(cfg)
+    ref = orc.run(cfg)
+    assert_same(cfg, gpu, ref, cfg.T_max, cfg.name)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+
+
+@pytest.mark.parametrize("cfg", scaled_presets(), ids=lambda c: c.name)
+def test_scaled_presets(cfg):
+    gpu = run_gpu(cfg)
+    ref = orc.run(cfg, threads=8)
+    assert_same(cfg, gpu, ref, cfg.T_max, cfg.name)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+
+
+def test_config1_full():
+    cfg = wl.config1()
+    gpu = run_gpu(cfg)
+    ref = orc.run(cfg, threads=8)
+    assert_same(cfg, gpu, ref, cfg.T_max, "cfg1")
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+
+
+@pytest.mark.parametrize("pieces", [[1] * 40 + [60], [33, 31, 36], [7, 64, 29], [99, 1]])
+def test_resumed_runs_equal_one_run(pieces):
+    for seed in (3, 11, 17):
+        cfg = wl.random_small_config(seed, n_replicas=4, T=100)
+        whole = run_gpu(cfg)
+        parts = run_gpu(cfg, pieces=pieces)
+        for k in ("counters", "trace", "hist", "complog"):
+            if whole[k] is not None:
+                assert (whole[k] == parts[k]).all(), (seed, k)
+    cfg = wl.config1(replicas=8, T=sum(pieces) * 10)
+    ref = orc.run(cfg)
+    parts = run_gpu(cfg, pieces=[p * 10 for p in pieces])
+    assert_same(cfg, parts, ref, cfg.T_max, "cfg1 resumed")
+
+
+def test_pause_counters_match_a_shorter_run():
+    cfg = wl.config5(replicas=4, T=3000)
+    gpu = run_gpu(cfg, n_steps=1234)
+    ref = orc.run(cfg, n_steps=1234)
+    assert_same(cfg, gpu, ref, 1234, "cfg5 paused")
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 1234)
+
+
+def test_more_replicas_than_resident_warps_and_many_groups():
+    # several replicas per warp (work queue), several launches, 24 groups
+    cfg = wl.config3(n_rates=4, n_b=6, reps=3, T=1500)
+    cfg = cfg.with_(Qcap=64, Acap=256)
+    gpu = run_gpu(cfg)
+    ref = orc.run(cfg, threads=8)
+    assert_same(cfg, gpu, ref, cfg.T_max, "cfg3 grid")
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+    big = wl.config1(replicas=20000, T=64).with_(trace_stride=8, complog_cap=8)
+    gpu = run_gpu(big)
+    ref = orc.run(big, threads=8)
+    assert_same(big, gpu, ref, big.T_max, "20000 replicas")
+
+
+def test_large_flow_rate_equals_greedy_on_gpu():
+    cfg = wl.config1(replicas=6, T=1200)
+    flow = cfg.with_(groups=(wl.Group(wl.POLICY_FLOW, b_fp=0xFFFF0000, n_replicas=6),))
+    greedy = cfg.with_(groups=(wl.Group(wl.POLICY_GREEDY, n_replicas=6),))
+    a, b = run_gpu(flow), run_gpu(greedy)
+    for k in ("trace", "hist", "complog"):
+        assert (a[k] == b[k]).all()
+    assert_same(flow, a, orc.run(flow), cfg.T_max, "flow b=65535")
+
+
+def test_edge_shapes():
+    # one replica; zero steps; tiny capacities (Acap blocks, waiting room of one); no outputs at all
+    one = degenerate_config(n=1, l=2, o=3, policy="flow", b=1, K=0, c=0, M=11, T=5)
+    gpu = run_gpu(one, n_steps=0)
+    assert (gpu["counters"] == 0).all()
+    tight = wl.config1(replicas=3, T=400).with_(Qcap=1, Acap=2, M=700)
+    assert_same(tight, run_gpu(tight), orc.run(tight), 400, "tight")
+    ref = orc.run(tight)
+    assert ref["counters"][:, orc.CIDX["acap_blocked_steps"]].sum() > 0
+    bare = wl.config1(replicas=3, T=300).with_(trace_stride=0, hist_bins=0, complog_cap=0)
+    assert_same(bare, run_gpu(bare), orc.run(bare), 300, "bare")
+    burst = degenerate_config(n=200, l=1, o=1, policy="greedy", b=0, K=0, c=0, M=100000, T=40, Qcap=1000, Acap=700)
+    assert_same(burst, run_gpu(burst), orc.run(burst), 40, "burst")
+    strided = wl.config1(replicas=2, T=1000).with_(trace_stride=7)
+    assert_same(strided, run_gpu(strided, pieces=[500, 3, 497]), orc.run(strided), 1000, "stride 7")
+
+
+def test_host_buffer_entry_point():
+    from paper_2604_11001_b200 import binding as fb
+    cfg = wl.config1(replicas=16, T=500)
+    out = fb.fcsim_simulate_host(cfg)
+    ref = orc.run(cfg)
+    assert_same(cfg, out, ref, 500, "simulate_host")
+    assert_summary_close(cfg, out["summary"], ref["counters"], ref["hist"], 500)
