@@ -133,7 +133,7 @@ def sized_oracle_sample(workload: int, slots: int, target_s: float):
     """Probe briefly, then run a sample sized to about target_s seconds of host time."""
     cores = os.cpu_count() or 1
     v, _, _, _ = oracle_sample(workload, slots, 2 * cores)
-    n = int(max(2 * cores, min(4096, v * target_s / slots)))
+    n = int(max(2 * cores, min(32768, v * target_s / slots)))
     return oracle_sample(workload, slots, n)
 
 
@@ -146,7 +146,7 @@ def run_reference(args):
     per_step_s = min(20.0, 150.0 / n_all)
     cores = os.cpu_count() or 1
     v, _, _, _ = oracle_sample(args.workload, slots, 2 * cores)
-    n = int(max(2 * cores, min(4096, v * per_step_s / slots)))
+    n = int(max(2 * cores, min(32768, v * per_step_s / slots)))
     times, vals, desc = [], [], ""
     for i in range(args.warmup + args.steps):
         v, cores, desc, dt = oracle_sample(args.workload, slots, n)
