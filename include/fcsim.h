@@ -37,7 +37,8 @@ enum {
     FCSIM_ESIZE = -3,  /* a required buffer is NULL or too small */
     FCSIM_ERANGE = -4, /* steps beyond T_max */
     FCSIM_ECUDA = -5,  /* CUDA runtime error; code via fcsim_last_cuda_error */
-    FCSIM_ENOMEM = -6  /* host allocation failed */
+    FCSIM_ENOMEM = -6, /* host allocation failed */
+    FCSIM_ETOOBIG = -7 /* fcsim_stats_noalloc: the group rows exceed the library's fixed device scratch */
 };
 
 enum { FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2 };
@@ -168,6 +169,32 @@ int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream);
  * host_out (HOST, [R], may be NULL) <- per-replica counters; per_group_out (HOST, [n_groups], may be
  * NULL) <- summaries. */
 int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_out, fcsim_summary* per_group_out);
+
+/* Group summaries for callers that must not allocate.  (The paper has no counterpart: this is a
+ * deployment convenience of the library.)
+ *
+ * Some hosts of this library cannot obtain device memory when they want statistics: a serving process
+ * whose memory manager has already claimed the whole GPU and hands none back, a monitoring thread that
+ * must not trigger the implicit device-wide synchronisation an allocation or free causes, or an embedding
+ * that simply forbids the CUDA allocator after start-up.  fcsim_stats needs a caller-allocated `scratch`
+ * buffer for its per-group rows; this variant needs none.  It runs the same two reduction kernels, but
+ * their group rows live in a fixed array inside the library's device image
+ * (FCSIM_NOALLOC_SCRATCH_WORDS 64-bit words = 1 MiB, held by every GPU that loads the library until the
+ * process exits), and the rows come back through a fixed host array inside the library.  It calls no
+ * device or host allocator and frees nothing.
+ *
+ * per_group_out: HOST, [n_groups], receives exactly what fcsim_stats would write there.
+ * Limit: n_groups * (28 + hist_bins) must not exceed FCSIM_NOALLOC_SCRATCH_WORDS, otherwise
+ * FCSIM_ETOOBIG is returned and nothing is launched.
+ * First call on a device: the library looks up the device address of its array (one runtime query, no
+ * allocation) and remembers it; make that first call outside any stream capture, with the handle's
+ * device current.
+ * Sharing: every call, from every handle, uses the one array; it still holds the previous call's rows,
+ * so each call clears the part it needs on `cuda_stream` before reducing.  Two calls whose GPU work
+ * overlaps (different streams or threads) race on the array and on the host staging array: serialise them.
+ * Synchronises `cuda_stream` before returning. */
+#define FCSIM_NOALLOC_SCRATCH_WORDS 131072
+int fcsim_stats_noalloc(fcsim_t* h, void* cuda_stream, fcsim_summary* per_group_out);
 
 int fcsim_destroy(fcsim_t* h);
 

@@ -73,7 +73,8 @@ class fcsim_launch_info(C.Structure):
 
 EXPORTS = ("fcsim_query_sizes", "fcsim_create", "fcsim_run", "fcsim_stats", "fcsim_destroy",
            "fcsim_steps_done", "fcsim_get_launch_info", "fcsim_last_cuda_error", "fcsim_last_cuda_error_name",
-           "fcsim_strerror", "fcsim_simulate_host", "fcsim_debug_read", "fcsim_is_checked_build")
+           "fcsim_strerror", "fcsim_simulate_host", "fcsim_debug_read", "fcsim_is_checked_build",
+           "fcsim_stats_noalloc")
 
 _lib = None
 
@@ -108,6 +109,7 @@ def load():
     lib.fcsim_last_cuda_error_name.restype = C.c_char_p
     lib.fcsim_debug_read.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.fcsim_is_checked_build.argtypes = []
+    lib.fcsim_stats_noalloc.argtypes = [vp, vp, C.POINTER(fcsim_summary)]
     for name in EXPORTS:
         if name not in ("fcsim_strerror", "fcsim_steps_done", "fcsim_last_cuda_error_name"):
             getattr(lib, name).restype = C.c_int
@@ -207,6 +209,20 @@ def fcsim_stats(handle: int, n_replicas: int, n_groups: int, stream=None, want_c
             d.update({n: float(getattr(s, n)) for n in SUMMARY_FLOATS})
             out.append(d)
     return cnt, out
+
+
+def fcsim_stats_noalloc(handle: int, n_groups: int, stream=None):
+    """Per-group summaries without any allocation by the library: for processes that cannot get device
+    memory any more (their allocator owns the GPU) or must not pay an allocation's device-wide stall.
+    The group rows use a fixed 1 MiB array inside the library, shared by all calls: do not overlap calls."""
+    summ = (fcsim_summary * n_groups)()
+    _check(load().fcsim_stats_noalloc(C.c_void_p(handle), _stream_ptr(stream), summ), "fcsim_stats_noalloc", handle)
+    out = []
+    for s in summ:
+        d = {n: int(getattr(s.total, n)) for n in COUNTER_NAMES}
+        d.update({n: float(getattr(s, n)) for n in SUMMARY_FLOATS})
+        out.append(d)
+    return out
 
 
 def fcsim_destroy(handle: int) -> None:

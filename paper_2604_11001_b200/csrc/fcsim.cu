@@ -456,6 +456,71 @@ extern "C" int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_o
     return FCSIM_OK;
 }
 
+// ---- statistics without any allocation --------------------------------------------------------------
+// For callers that cannot allocate device memory (a process whose allocator already owns the whole GPU,
+// a thread that must avoid the device-wide synchronisation of cudaMalloc/cudaFree).  The per-group rows
+// that fcsim_stats keeps in the caller's scratch buffer live here in a fixed array of the device image.
+// On the host the array's name is only a stand-in for the symbol, never a device address: its address
+// on the current device is queried once per device with cudaGetSymbolAddress and that pointer is what
+// the kernels get.
+static __device__ __align__(256) long long g_noalloc_scratch[FCSIM_NOALLOC_SCRATCH_WORDS];
+static long long g_noalloc_host_rows[FCSIM_NOALLOC_SCRATCH_WORDS];   // host staging for the copy back
+constexpr int kNoallocMaxDevices = 64;
+static long long* g_noalloc_dev_ptr[kNoallocMaxDevices] = {nullptr};
+
+extern "C" int fcsim_stats_noalloc(fcsim_t* h, void* cuda_stream, fcsim_summary* per_group_out) {
+    if (!h || !per_group_out) return FCSIM_EINVAL;
+    const int G = (int)h->groups.size();
+    const int bins = h->cfg.hist_bins;
+    const int R = (int)h->L.R;
+    const size_t words = (size_t)G * ((size_t)C_COUNT + (size_t)bins);
+    if (words > (size_t)FCSIM_NOALLOC_SCRATCH_WORDS) return FCSIM_ETOOBIG;
+    int dev = -1;
+    CUDA_TRY(h, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kNoallocMaxDevices || dev != h->device) return FCSIM_EINVAL;
+    if (!g_noalloc_dev_ptr[dev]) {   // set-up, once per device, with that device current
+        void* sym = nullptr;
+        CUDA_TRY(h, cudaGetSymbolAddress(&sym, g_noalloc_scratch));
+        g_noalloc_dev_ptr[dev] = static_cast<long long*>(sym);
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    long long* d_cnt = g_noalloc_dev_ptr[dev];
+    long long* d_hist = d_cnt + (size_t)G * C_COUNT;
+    // the array still holds the rows of the previous call: the sums must start from zero
+    CUDA_TRY(h, cudaMemsetAsync(d_cnt, 0, words * 8, st));
+    const int n_chunks = (R + kStatsChunk - 1) / kStatsChunk;
+    {
+        const int warps_per_block = 8;
+        const int blocks = std::max(1, std::min((n_chunks + warps_per_block - 1) / warps_per_block, h->sm_count * 8));
+        reduce_counters_kernel<<<blocks, warps_per_block * 32, 0, st>>>(
+            static_cast<const long long*>(h->buf.counters), h->d_groups, G, R, kStatsChunk, d_cnt);
+        CUDA_TRY(h, cudaGetLastError());
+    }
+    if (bins > 0) {
+        const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
+        reduce_hist_kernel<<<blocks, 256, 0, st>>>(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins,
+                                                   kStatsChunk, d_hist);
+        CUDA_TRY(h, cudaGetLastError());
+    }
+    CUDA_TRY(h, cudaMemcpyAsync(g_noalloc_host_rows, d_cnt, words * 8, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(h, cudaStreamSynchronize(st));
+    const double T = (double)h->t_done;
+    for (int g = 0; g < G; ++g) {
+        fcsim_summary& s = per_group_out[g];
+        std::memcpy(&s.total, g_noalloc_host_rows + (size_t)g * C_COUNT, sizeof(fcsim_counters));
+        const double n = (double)h->groups[g].n_replicas;
+        const fcsim_counters& c = s.total;
+        s.mean_latency = c.completed > 0 ? (double)c.sum_lat / (double)c.completed : 0.0;
+        s.mean_utilisation = T > 0 ? (double)c.sum_U / (n * T * (double)h->cfg.M) : 0.0;
+        s.request_throughput = T > 0 ? (double)c.completed / (n * T) : 0.0;
+        s.token_throughput = T > 0 ? (double)c.tokens_generated / (n * T) : 0.0;
+        const long long* gh = g_noalloc_host_rows + (size_t)G * C_COUNT + (size_t)g * bins;
+        s.p95_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 95, c.max_lat);
+        s.p99_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 99, c.max_lat);
+    }
+    return FCSIM_OK;
+}
+
 extern "C" int fcsim_destroy(fcsim_t* h) {
     if (!h) return FCSIM_EINVAL;
     release(h);
@@ -506,6 +571,7 @@ extern "C" const char* fcsim_strerror(int code) {
         case FCSIM_ERANGE: return "steps beyond T_max";
         case FCSIM_ECUDA: return "CUDA runtime error";
         case FCSIM_ENOMEM: return "host allocation failed";
+        case FCSIM_ETOOBIG: return "group rows exceed the fixed device scratch of fcsim_stats_noalloc";
         default: return "unknown error";
     }
 }
