@@ -84,7 +84,9 @@ def load():
     global _lib
     if _lib is not None:
         return _lib
-    if os.environ.get("FCSIM_CHECKED"):     # index-checked diagnostic build
+    if os.environ.get("FCSIM_LIB"):           # explicit library path (diagnostic builds)
+        path = os.environ["FCSIM_LIB"]
+    elif os.environ.get("FCSIM_CHECKED"):     # index-checked diagnostic build
         path = _build.LIB_CHECKED if os.path.exists(_build.LIB_CHECKED) else _build.build(checked=True)
     else:
         path = _build.LIB

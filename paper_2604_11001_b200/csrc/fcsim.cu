@@ -189,6 +189,7 @@ struct fcsim {
     fcsim_buffers buf;
     Params params;
     uint32_t* d_pool = nullptr;
+    unsigned short* d_gpool = nullptr;
     DevTable* d_tables = nullptr;
     DevArrivals* d_arrivals = nullptr;
     DevGroup* d_groups = nullptr;
@@ -219,13 +220,28 @@ extern "C" int fcsim_query_sizes(const fcsim_config* cfg, fcsim_sizes* out) {
 
 static int upload_tables(fcsim* h, const fcsim_config* c) {
     std::vector<uint32_t> pool;
+    std::vector<unsigned short> gpool(2, 0);  // offset 0 is never a guide
     auto add = [&](const fcsim_table& t) {
         DevTable d;
         d.off = (uint32_t)pool.size();
         d.n = t.n;
         d.vmin = t.vmin;
-        d.pad = 0;
+        d.guide = 0;
         pool.insert(pool.end(), t.cdf, t.cdf + t.n);
+        if (t.n >= 16) {
+            // guide[b] = first k < n-1 with cdf[k] > (b << shift), else n-1; guide[2^bits] = n-1
+            uint32_t bits = 4;
+            while (bits < 10 && (4u << bits) < t.n) ++bits;
+            const uint32_t shift = 32 - bits;
+            d.guide = (bits << 27) | (uint32_t)gpool.size();
+            uint32_t k = 0;
+            for (uint32_t b = 0; b < (1u << bits); ++b) {
+                const uint32_t edge = b << shift;
+                while (k < t.n - 1 && t.cdf[k] <= edge) ++k;
+                gpool.push_back((unsigned short)k);
+            }
+            gpool.push_back((unsigned short)(t.n - 1));
+        }
         return d;
     };
     std::vector<DevTable> tables;
@@ -249,6 +265,8 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas, 0};
         first += G.n_replicas;
     }
+    CUDA_TRY(h, cudaMalloc(&h->d_gpool, gpool.size() * sizeof(unsigned short)));
+    CUDA_TRY(h, cudaMemcpy(h->d_gpool, gpool.data(), gpool.size() * sizeof(unsigned short), cudaMemcpyHostToDevice));
     CUDA_TRY(h, cudaMalloc(&h->d_pool, pool.size() * sizeof(uint32_t)));
     CUDA_TRY(h, cudaMalloc(&h->d_tables, tables.size() * sizeof(DevTable)));
     CUDA_TRY(h, cudaMalloc(&h->d_arrivals, arrs.size() * sizeof(DevArrivals)));
@@ -267,6 +285,7 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
 static void release(fcsim* h) {
     if (!h) return;
     cudaFree(h->d_pool);
+    cudaFree(h->d_gpool);
     cudaFree(h->d_tables);
     cudaFree(h->d_arrivals);
     cudaFree(h->d_groups);
@@ -350,6 +369,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.n_classes = cfg->n_classes; p.n_groups = cfg->n_groups; p.n_replicas = (int)L.R;
     p.trace_stride = cfg->trace_stride; p.n_rec = L.n_rec;
     p.hist_bins = cfg->hist_bins; p.hist_shift = cfg->hist_shift; p.complog_cap = cfg->complog_cap;
+    p.gpool = h->d_gpool;
     p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
     p.workspace = static_cast<unsigned char*>(b->workspace);
     p.ws_stride = L.ws_stride;

@@ -13,7 +13,9 @@
 //                      prompt is in the cache the slot in which its last token is generated
 //                      (t_fin = activation slot + o - 1, so its output count is implied by the
 //                      slot number and "process all requests" costs nothing); for a request still
-//                      prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so far.
+//                      prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so far;
+//                      0 for a request that has completed but whose entry has not been squeezed
+//                      out yet (completed entries are removed lazily, many at a time).
 //   stage [S]    u64   arrivals generated ahead of time for the next batch of <= 32 slots.
 #pragma once
 #include <cstdint>
@@ -25,6 +27,8 @@ constexpr int kWarpsPerBlock = 4;
 constexpr int kHeaderWords = 16;  // per-replica scalar state kept in the workspace
 constexpr uint32_t kNoFin = 0xFFFFFFFFu;
 constexpr uint32_t kPrefillBit = 0x80000000u;
+constexpr uint32_t kDead = 0u;        // state word of a completed entry awaiting removal
+constexpr int kCompactAt = 32;        // completed entries tolerated inside the active range
 
 enum CounterIdx {
     C_STEPS_DONE = 0, C_STATUS, C_ARRIVED, C_DROPPED, C_ADMITTED, C_COMPLETED, C_EVICTIONS,
@@ -38,7 +42,7 @@ struct DevTable {
     uint32_t off;  // first threshold in the pool
     uint32_t n;
     int32_t vmin;
-    uint32_t pad;
+    uint32_t guide;  // bits 27..31: log2 of the guide size (0 = no guide); bits 0..26: offset in the guide pool
 };
 struct DevArrivals {
     DevTable count[2];
@@ -64,6 +68,7 @@ struct Params {
     int32_t trace_stride, n_rec, hist_bins, hist_shift, complog_cap;
     int32_t t0, n_steps;
     const uint32_t* pool;         // all thresholds
+    const unsigned short* gpool;  // guide tables: for bucket b of the top bits of u, the first candidate index
     const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
     const DevArrivals* arrivals;
     const DevGroup* groups;
@@ -95,10 +100,20 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     o0 = c0; o1 = c1; o2 = c2; o3 = c3;
 }
 
-// vmin + (first k < n-1 with thresholds[k] > u, else n-1).
-__device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, const DevTable tb, uint32_t u) {
+// vmin + (first k < n-1 with thresholds[k] > u, else n-1).  A guide table indexed by the top bits of u
+// brackets the answer (entry b = first index whose threshold exceeds b << shift), so the binary search
+// runs over a few entries instead of the whole table.
+__device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, const unsigned short* __restrict__ gpool,
+                                            const DevTable tb, uint32_t u) {
     const uint32_t* __restrict__ cdf = pool + tb.off;
     uint32_t lo = 0, hi = tb.n - 1;
+    const uint32_t gbits = tb.guide >> 27;
+    if (gbits) {
+        const unsigned short* __restrict__ g = gpool + (tb.guide & 0x7ffffffu);
+        const uint32_t b = u >> (32u - gbits);
+        lo = __ldg(g + b);
+        hi = __ldg(g + b + 1);
+    }
     while (lo < hi) {
         const uint32_t mid = (lo + hi) >> 1;
         if (__ldg(cdf + mid) > u) hi = mid; else lo = mid + 1;
@@ -106,6 +121,11 @@ __device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, c
     return tb.vmin + (int)lo;
 }
 
+__device__ __forceinline__ uint32_t lanemask_lt() {
+    uint32_t m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
 __device__ __forceinline__ uint32_t lanemask_gt() {
     uint32_t m;
     asm("mov.u32 %0, %%lanemask_gt;" : "=r"(m));
@@ -165,7 +185,12 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define HROW(i) hrow[(i)]
 #endif
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const Params p) {
+// Minimum resident CTAs per SM the compiler must allow for (bounds registers per thread).
+#ifndef FCSIM_MIN_CTAS
+#define FCSIM_MIN_CTAS 5
+#endif
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_step_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -179,6 +204,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
     const bool kinf = (K == 0);
     const uint32_t FULL = 0xffffffffu;
     const uint32_t gt_mask = lanemask_gt();
+    const uint32_t lt_mask = lanemask_lt();
 
     for (;;) {
         // ------------------------------------------------------------------ next replica
@@ -197,19 +223,22 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
             gi = lo;
         }
         const DevGroup grp = p.groups[gi];
-        const DevArrivals arr = p.arrivals[grp.arrivals_id];
+        const DevArrivals* arrp = p.arrivals + grp.arrivals_id;
+        const DevTable cnt0 = arrp->count[0];
+        const DevTable cnt1 = arrp->count[1];
+        const uint32_t thr0 = arrp->thr[0], thr1 = arrp->thr[1];
+        const bool two_state = arrp->n_states == 2;
         const uint32_t rid = grp.rng_base + (r - (unsigned)grp.first);
         const int policy = grp.policy;
         const int chunk = grp.chunk;
-        const bool two_state = arr.n_states == 2;
 
         // ------------------------------------------------------------------ load state
         unsigned char* ws = p.workspace + (size_t)r * p.ws_stride;
         uint32_t* hdr = reinterpret_cast<uint32_t*>(ws);
         const uint32_t hw = (lane < kHeaderWords) ? hdr[lane] : 0u;
-        int head = (int)__shfl_sync(FULL, hw, 0);
-        int shead = (int)__shfl_sync(FULL, hw, 1);
-        int nP = (int)__shfl_sync(FULL, hw, 2);
+        int head = (int)__shfl_sync(FULL, hw, 0);     // ring position of the oldest active entry
+        int shead = (int)__shfl_sync(FULL, hw, 1);    // same for the state ring
+        int nP = (int)__shfl_sync(FULL, hw, 2);       // entries in the active range, completed ones included
         int nQ = (int)__shfl_sync(FULL, hw, 3);
         int U = (int)__shfl_sync(FULL, hw, 4);        // usage carried out of the last slot, completions released
         int Ndec = (int)__shfl_sync(FULL, hw, 5);     // active requests whose prompt is fully in the cache
@@ -218,6 +247,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
         int pf_lo = (int)__shfl_sync(FULL, hw, 8);    // lower bound on the index of the oldest of those
         uint32_t mstate = __shfl_sync(FULL, hw, 9);
         uint32_t status = __shfl_sync(FULL, hw, 10);
+        int nD = (int)__shfl_sync(FULL, hw, 11);      // completed entries still inside the active range
         {
             const uint4* src = reinterpret_cast<const uint4*>(ws + kHeaderWords * 4);
             uint4* dst = reinterpret_cast<uint4*>(my);
@@ -236,9 +266,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
 
         // per-launch partial sums of the quantities touched every slot
         unsigned long long sumU = 0;
-        uint32_t sumN = 0, tokgen = 0, arrived = 0;
+        uint32_t sumN = 0, tokgen = 0, arrived = 0, dropped = 0;
         int maxU = 0, maxQ = 0;
         int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
+        int q_l = -1;  // prompt length of the queue head when known (saves a shared-memory read per blocked slot)
 
         int t = p.t0;
         const int t_end = p.t0 + p.n_steps;
@@ -253,22 +284,58 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
         int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
         int2* lrow = p.complog ? p.complog + (size_t)r * p.complog_cap : nullptr;
 
+        // Squeeze the completed entries out of the active range: survivors slide towards the queue
+        // boundary (right-to-left pass), the head advances, the queue is not touched.
+        auto compact = [&]() {
+            int holes = 0;
+            for (int base = (nP - 1) & ~31; base >= 0; base -= 32) {
+                const int i = base + lane;
+                const bool valid = i < nP;
+                uint32_t sw = kDead;
+                uint64_t e = 0;
+                if (valid) sw = STATE(WA(shead + i));
+                const bool dead = valid && (sw == kDead);
+                const uint32_t m = __ballot_sync(FULL, dead);
+                const int sh = holes + __popc(m & gt_mask);  // completed entries after this one
+                const bool mv = valid && !dead && sh > 0;
+                if (mv) e = RING(WR(head + i));
+                __syncwarp();
+                if (mv) {
+                    RING(WR(head + i + sh)) = e;
+                    STATE(WA(shead + i + sh)) = sw;
+                }
+                __syncwarp();
+                holes += __popc(m);
+            }
+            head = WR(head + nD);
+            shead = WA(shead + nD);
+            nP -= nD;
+            pf_lo = max(0, pf_lo - nD);
+            nD = 0;
+        };
+
         while (t < t_end) {
             // -------------------------------------------------------------- batch: draws of up to 32 slots
             int L = min(32, t_end - t);
             uint32_t w0, w1, w2, w3;
             philox4x32_10((uint32_t)(t + 1 + lane), rid, 0u, 0u, p.key0, p.key1, w0, w1, w2, w3);
             const int Bt = (int)(grp.b_fp >> 16) + (((w1 >> 16) < (grp.b_fp & 0xffffu)) ? 1 : 0);
-            int n = sample_table(p.pool, arr.count[0], w0);
+            int n = sample_table(p.pool, p.gpool, cnt0, w0);
             uint32_t smask = 0;  // bit k = arrival state in slot t+1+k
             if (two_state) {
-                const int n1 = sample_table(p.pool, arr.count[1], w0);
-                const uint32_t f0 = __ballot_sync(FULL, w2 < arr.thr[0]);
-                const uint32_t f1 = __ballot_sync(FULL, w2 < arr.thr[1]);
-                uint32_t cur = mstate;
-                for (int k = 0; k < 32; ++k) {
-                    cur ^= ((cur ? f1 : f0) >> k) & 1u;
-                    smask |= cur << k;
+                const int n1 = sample_table(p.pool, p.gpool, cnt1, w0);
+                const uint32_t f0 = __ballot_sync(FULL, w2 < thr0);
+                const uint32_t f1 = __ballot_sync(FULL, w2 < thr1);
+                if (f0 == f1) {  // same flips from either state: parity of the flips so far
+                    const uint32_t upto = f0 & (lt_mask | (1u << lane));
+                    const uint32_t mine = (mstate ^ (uint32_t)__popc(upto)) & 1u;
+                    smask = __ballot_sync(FULL, mine != 0u);
+                } else {
+                    uint32_t cur = mstate;
+                    for (int k = 0; k < 32; ++k) {
+                        cur ^= ((cur ? f1 : f0) >> k) & 1u;
+                        smask |= cur << k;
+                    }
                 }
                 if ((smask >> lane) & 1u) n = n1;
             }
@@ -293,32 +360,35 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                     uint32_t a0, a1, a2, a3;
                     philox4x32_10((uint32_t)(t + 1 + lo), rid, 1u, (uint32_t)(idx - ex_k), p.key0, p.key1, a0, a1,
                                   a2, a3);
-                    const int cls = sample_table(p.pool, p.tables[0], a0);
-                    const int l = sample_table(p.pool, p.tables[1 + cls], a1);
-                    const int o = sample_table(p.pool, p.tables[1 + p.n_classes + cls], a2);
+                    const int cls = sample_table(p.pool, p.gpool, p.tables[0], a0);
+                    const int l = sample_table(p.pool, p.gpool, p.tables[1 + cls], a1);
+                    const int o = sample_table(p.pool, p.gpool, p.tables[1 + p.n_classes + cls], a2);
                     STAGE(idx) = pack_entry(l, o, t + 1 + lo, cls);
                 }
             }
             __syncwarp();
             const uint32_t packed = (uint32_t)n | ((uint32_t)Bt << 8);
+            int sp = 0;  // staged arrivals consumed so far
 
             // -------------------------------------------------------------- the slots of the batch
             for (int k = 0; k < L; ++k) {
                 ++t;
                 const uint32_t info = __shfl_sync(FULL, packed, k);
-                const int ex = __shfl_sync(FULL, excl, k);
                 const int n_t = (int)(info & 0xffu);
                 const int B_t = (int)(info >> 8);
 
                 // ---- arrivals join the queue tail; a full waiting room drops the rest
                 if (n_t > 0) {
                     const int acc = min(n_t, max(0, Qcap - nQ));
-                    const int tail = head + nP + nQ;
-                    for (int i = lane; i < acc; i += 32) RING(WR(WR(tail) + i)) = STAGE(ex + i);
-                    nQ += acc;
+                    if (acc > 0) {
+                        const int tail = WR(head + nP + nQ);
+                        for (int i = lane; i < acc; i += 32) RING(WR(tail + i)) = STAGE(sp + i);
+                        nQ += acc;
+                        __syncwarp();
+                    }
+                    sp += n_t;
                     arrived += n_t;
-                    if (acc < n_t) CADD(C_DROPPED, n_t - acc);
-                    __syncwarp();
+                    dropped += n_t - acc;
                 }
 
                 // ---- usage the slot would reach, token room
@@ -332,8 +402,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                         const int i = base + lane;
                         uint32_t sw = 0;
                         uint64_t e = 0;
-                        if (i < nP) { sw = STATE(WA(shead + i)); e = RING(WR(head + i)); }
+                        if (i < nP) sw = STATE(WA(shead + i));
                         const bool pf = (sw & kPrefillBit) != 0;
+                        if (pf) e = RING(WR(head + i));
                         const int pcur = (int)(sw & ~kPrefillBit);
                         const int l = entry_l(e);
                         const int d = pf ? min(chunk, l - pcur) : 0;
@@ -364,14 +435,18 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                     __syncwarp();
                 }
 
+                // ---- completed entries must be gone before an eviction (the newest entry has to be a live
+                //      one), before the active range runs out of storage, and when too many have piled up
+                if (nD > 0 && (nD >= kCompactAt || G > M || nP + nQ > Acap)) compact();
+
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
                 {
                     int a = 0;
                     const int cap = (policy == 0) ? B_t : 0x7fffffff;
                     while (a < cap && nQ > 0) {
                         if (nP == Acap) { CADD(C_ACAP_BLOCKED, 1); status |= 1u; break; }
-                        const uint64_t e = RING(WR(head + nP));
-                        const int l = entry_l(e);
+                        if (q_l < 0) q_l = entry_l(RING(WR(head + nP)));
+                        const int l = q_l;
                         int g, need;
                         if (policy == 2) {
                             g = kinf ? min(chunk, l) : min(min(chunk, l), R);
@@ -385,7 +460,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                         if (G + need > M) { CADD(C_GATE_BLOCKED, 1); break; }
                         uint32_t sw;
                         if (g == l) {
-                            sw = (uint32_t)(t + entry_o(e) - 1);
+                            sw = (uint32_t)(t + entry_o(RING(WR(head + nP))) - 1);
                             next_fin = min(next_fin, sw);
                             Ndec++;
                         } else {
@@ -396,6 +471,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                         if (lane == 0) STATE(WA(shead + nP)) = sw;
                         nP++;
                         nQ--;
+                        q_l = -1;
                         G += need;
                         if (!kinf) R -= min(g, R);
                         a++;
@@ -412,16 +488,17 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                     while (G > M && nP > 0) {
                         const int i = nP - 1;
                         const uint32_t sw = STATE(WA(shead + i));
+                        const uint64_t e = RING(WR(head + i));
                         if (sw & kPrefillBit) {
                             G -= (int)(sw & ~kPrefillBit);
                             n_pref--;
                         } else {
-                            const uint64_t e = RING(WR(head + i));
                             const int j = t - (int)sw + entry_o(e) - 1;  // tokens generated before this slot
                             G -= entry_l(e) + j + 1;
                             wasted += j;
                             Ndec--;
                         }
+                        q_l = entry_l(e);
                         nP--;
                         nQ++;
                         nev++;
@@ -436,35 +513,23 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                 U = G;
                 sumU += (unsigned)G;
                 maxU = max(maxU, G);
-                sumN += nP + nQ;
+                sumN += nP - nD + nQ;
 
-                // ---- retire the requests that generated their last token in this slot
+                // ---- retire the requests that generated their last token in this slot: their statistics
+                //      are taken now, their entries are only marked and squeezed out later in bulk
                 if ((uint32_t)t == next_fin) {
                     uint32_t newmin = kNoFin;
-                    int ndone = 0, top = -1;
+                    int ndone = 0;
+                    int sum_lat = 0, sum_o = 0, sum_lo = 0, max_lat = 0;
+                    long long sum_w = 0;
                     for (int base = 0; base < nP; base += 32) {
                         const int i = base + lane;
-                        const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kNoFin;
+                        const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
                         const bool done = (sw == (uint32_t)t);
                         const uint32_t m = __ballot_sync(FULL, done);
-                        if (m) { ndone += __popc(m); top = base + 31 - __clz(m); }
-                        if (!done) newmin = min(newmin, sw);
-                    }
-                    next_fin = __reduce_min_sync(FULL, newmin);
-                    if (ndone > 0) {
-                        int holes = 0;  // completions at higher indices than the current block
-                        int sum_lat = 0, sum_o = 0, sum_lo = 0, max_lat = 0;
-                        long long sum_w = 0;
-                        for (int base = top & ~31; base >= 0; base -= 32) {
-                            const int i = base + lane;
-                            const bool valid = i <= top;
-                            uint32_t sw = kNoFin;
-                            uint64_t e = 0;
-                            if (valid) { sw = STATE(WA(shead + i)); e = RING(WR(head + i)); }
-                            const bool done = valid && (sw == (uint32_t)t);
-                            const uint32_t m = __ballot_sync(FULL, done);
-                            const int sh = holes + __popc(m & gt_mask);  // completions after this entry
+                        if (m) {
                             if (done) {
+                                const uint64_t e = RING(WR(head + i));
                                 const int l = entry_l(e), o = entry_o(e);
                                 const int lat = t - entry_tarr(e) + 1;
                                 sum_lat += lat;
@@ -474,34 +539,31 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
                                 sum_w += (long long)l * o + (long long)o * (o + 1) / 2;
                                 if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
                                 if (lrow) {
-                                    const int li = n_logged + ndone - 1 - sh;  // log is in activation order
+                                    const int li = n_logged + ndone + __popc(m & lt_mask);  // activation order
                                     if (li < p.complog_cap) LROW(li) = make_int2(t, lat);
                                 }
+                                STATE(WA(shead + i)) = kDead;
                             }
-                            __syncwarp();
-                            if (valid && !done && sh > 0) {  // survivors slide up over the holes
-                                RING(WR(head + i + sh)) = e;
-                                STATE(WA(shead + i + sh)) = sw;
-                            }
-                            __syncwarp();
-                            holes += __popc(m);
+                            ndone += __popc(m);
                         }
-                        head = WR(head + ndone);
-                        shead = WA(shead + ndone);
-                        nP -= ndone;
+                        const uint32_t cand = (done || sw == kDead) ? kNoFin : sw;
+                        newmin = min(newmin, cand);
+                    }
+                    next_fin = __reduce_min_sync(FULL, newmin);
+                    if (ndone > 0) {
+                        nD += ndone;
                         Ndec -= ndone;
-                        pf_lo = max(0, pf_lo - ndone);
                         U -= __reduce_add_sync(FULL, sum_lo);
                         CADD(C_COMPLETED, ndone);
                         CADD(C_SUM_LAT, __reduce_add_sync(FULL, sum_lat));
                         CADD(C_COMPLETED_TOKENS, __reduce_add_sync(FULL, sum_o));
                         CMAX(C_MAX_LAT, __reduce_max_sync(FULL, max_lat));
-                        const long long sw_all = warp_sum64(sum_w);
-                        CADD(C_SUM_W_COMPLETED, sw_all);
+                        CADD(C_SUM_W_COMPLETED, warp_sum64(sum_w));
                         if (lrow) {
                             if (n_logged + ndone > p.complog_cap) status |= 2u;
                             n_logged = min(p.complog_cap, n_logged + ndone);
                         }
+                        __syncwarp();
                     }
                 }
 
@@ -528,11 +590,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
         long long age = 0, resj = 0;
         for (int i = lane; i < nP + nQ; i += 32) {
             const uint64_t e = RING(WR(head + i));
-            age += t_end - entry_tarr(e) + 1;
+            bool live = true;
             if (i < nP) {
                 const uint32_t sw = STATE(WA(shead + i));
-                if (!(sw & kPrefillBit)) resj += t_end - (int)sw + entry_o(e);
+                live = (sw != kDead);
+                if (live && !(sw & kPrefillBit)) resj += t_end - (int)sw + entry_o(e);
             }
+            if (live) age += t_end - entry_tarr(e) + 1;
         }
         age = warp_sum64(age);
         resj = warp_sum64(resj);
@@ -540,13 +604,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
         CADD(C_SUM_N, sumN);
         CADD(C_TOKENS_GENERATED, tokgen);
         CADD(C_ARRIVED, arrived);
+        CADD(C_DROPPED, dropped);
         CMAX(C_MAX_U, maxU);
         CMAX(C_MAX_Q, maxQ);
         CSET(C_STEPS_DONE, t_end);
         CSET(C_STATUS, status);
         CSET(C_N_LOGGED, n_logged);
         CSET(C_Q_FINAL, nQ);
-        CSET(C_P_FINAL, nP);
+        CSET(C_P_FINAL, nP - nD);
         CSET(C_RESID_AGE, age);
         CSET(C_RESID_J, resj);
         CSET(C_MMPP_STATE, mstate);
@@ -565,6 +630,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fcsim_step_kernel(const P
             case 8: out = (uint32_t)pf_lo; break;
             case 9: out = mstate; break;
             case 10: out = status; break;
+            case 11: out = (uint32_t)nD; break;
             default: break;
         }
         if (lane < kHeaderWords) hdr[lane] = out;
