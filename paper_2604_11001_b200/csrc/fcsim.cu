@@ -81,7 +81,7 @@ int plan(const fcsim_config* c, Layout* L) {
     if (rc > (1 << 20)) return FCSIM_ECAP;
     L->RC = (int)align_up((size_t)rc, 2);
     L->Apad = (int)align_up((size_t)c->Acap, 4);
-    L->S = (int)align_up((size_t)std::max(64, max_count), 2);
+    L->S = (int)align_up((size_t)std::max(128, max_count), 2);
     L->ws_stride = kHeaderWords * 4 + (size_t)L->RC * 8 + (size_t)L->Apad * 4;
     L->smem_per_warp = (size_t)L->RC * 8 + (size_t)L->Apad * 4 + (size_t)L->S * 8;
     if (L->smem_per_warp > kSmemBudget) return FCSIM_ECAP;

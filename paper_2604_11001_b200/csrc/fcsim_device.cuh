@@ -205,6 +205,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
     const uint32_t FULL = 0xffffffffu;
     const uint32_t gt_mask = lanemask_gt();
     const uint32_t lt_mask = lanemask_lt();
+    int bsh = 5;  // lane c watches the entries [c << bsh, (c+1) << bsh) of the active range
+    while ((32 << bsh) < Acap) ++bsh;
 
     for (;;) {
         // ------------------------------------------------------------------ next replica
@@ -270,6 +272,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
         int maxU = 0, maxQ = 0;
         int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
         int q_l = -1;  // prompt length of the queue head when known (saves a shared-memory read per blocked slot)
+        // statistics of completions, private to the lane that saw them; reduced once when the replica is put back
+        unsigned long long acc_lat = 0, acc_w = 0;
+        uint32_t acc_o = 0, completed = 0;
+        int acc_maxlat = 0;
+        // cmin: lane c holds a lower bound of the smallest finishing slot among its stretch of the active
+        // range (exact except after an eviction, which a later rescan repairs)
+        uint32_t cmin = kNoFin;
 
         int t = p.t0;
         const int t_end = p.t0 + p.n_steps;
@@ -313,6 +322,18 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
             pf_lo = max(0, pf_lo - nD);
             nD = 0;
         };
+        // block minima of the finishing slots, from scratch
+        auto rebuild_minima = [&]() {
+            cmin = kNoFin;
+            for (int base = 0; base < nP; base += 32) {
+                const int i = base + lane;
+                const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
+                const uint32_t m = __reduce_min_sync(FULL, sw == kDead ? kNoFin : sw);
+                if (lane == (base >> bsh)) cmin = min(cmin, m);
+            }
+            next_fin = __reduce_min_sync(FULL, cmin);
+        };
+        rebuild_minima();
 
         while (t < t_end) {
             // -------------------------------------------------------------- batch: draws of up to 32 slots
@@ -398,7 +419,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                 // ---- chunked policy: continuing prefills first, in activation order
                 if (policy == 2 && n_pref > 0) {
                     int first_left = -1;
-                    for (int base = pf_lo; base < nP; base += 32) {
+                    for (int base = pf_lo & ~31; base < nP; base += 32) {
                         const int i = base + lane;
                         uint32_t sw = 0;
                         uint64_t e = 0;
@@ -426,7 +447,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                         n_pref -= nfin;
                         if (finm) {
                             const uint32_t mine = fin ? (uint32_t)(t + entry_o(e) - 1) : kNoFin;
-                            next_fin = min(next_fin, __reduce_min_sync(FULL, mine));
+                            const uint32_t bm = __reduce_min_sync(FULL, mine);
+                            if (lane == (base >> bsh)) cmin = min(cmin, bm);
+                            next_fin = min(next_fin, bm);
                         }
                         if (first_left < 0 && leftm) first_left = base + (__ffs(leftm) - 1);
                         if (!kinf && R == 0 && first_left >= 0) break;  // nothing more can move this slot
@@ -437,14 +460,18 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
 
                 // ---- completed entries must be gone before an eviction (the newest entry has to be a live
                 //      one), before the active range runs out of storage, and when too many have piled up
-                if (nD > 0 && (nD >= kCompactAt || G > M || nP + nQ > Acap)) compact();
+                bool squeeze = nD > 0 && (nD >= kCompactAt || G > M);
 
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
-                {
-                    int a = 0;
-                    const int cap = (policy == 0) ? B_t : 0x7fffffff;
+                int a = 0;
+                const int cap = (policy == 0) ? B_t : 0x7fffffff;
+                for (;;) {
+                    if (squeeze) { compact(); rebuild_minima(); squeeze = false; }
                     while (a < cap && nQ > 0) {
-                        if (nP == Acap) { CADD(C_ACAP_BLOCKED, 1); status |= 1u; break; }
+                        if (nP == Acap) {
+                            if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room
+                            CADD(C_ACAP_BLOCKED, 1); status |= 1u; break;
+                        }
                         if (q_l < 0) q_l = entry_l(RING(WR(head + nP)));
                         const int l = q_l;
                         int g, need;
@@ -462,6 +489,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                         if (g == l) {
                             sw = (uint32_t)(t + entry_o(RING(WR(head + nP))) - 1);
                             next_fin = min(next_fin, sw);
+                            if (lane == (nP >> bsh)) cmin = min(cmin, sw);
                             Ndec++;
                         } else {
                             sw = kPrefillBit | (uint32_t)g;
@@ -477,8 +505,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                         a++;
                         CADD(C_PREFILL_TOKENS, g);
                     }
-                    if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
+                    if (!squeeze) break;
                 }
+                if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
 
                 // ---- overflow: evict the most recently activated until the slot fits (LIFO, Section 3.3);
                 //      evicted requests lose all progress and are again the head of the queue
@@ -518,47 +547,47 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                 // ---- retire the requests that generated their last token in this slot: their statistics
                 //      are taken now, their entries are only marked and squeezed out later in bulk
                 if ((uint32_t)t == next_fin) {
-                    uint32_t newmin = kNoFin;
-                    int ndone = 0;
-                    int sum_lat = 0, sum_o = 0, sum_lo = 0, max_lat = 0;
-                    long long sum_w = 0;
-                    for (int base = 0; base < nP; base += 32) {
-                        const int i = base + lane;
-                        const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
-                        const bool done = (sw == (uint32_t)t);
-                        const uint32_t m = __ballot_sync(FULL, done);
-                        if (m) {
-                            if (done) {
-                                const uint64_t e = RING(WR(head + i));
-                                const int l = entry_l(e), o = entry_o(e);
-                                const int lat = t - entry_tarr(e) + 1;
-                                sum_lat += lat;
-                                sum_o += o;
-                                sum_lo += l + o;
-                                max_lat = max(max_lat, lat);
-                                sum_w += (long long)l * o + (long long)o * (o + 1) / 2;
-                                if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
-                                if (lrow) {
-                                    const int li = n_logged + ndone + __popc(m & lt_mask);  // activation order
-                                    if (li < p.complog_cap) LROW(li) = make_int2(t, lat);
+                    int ndone = 0, sum_lo = 0;
+                    uint32_t due = __ballot_sync(FULL, cmin == (uint32_t)t);
+                    while (due) {
+                        const int c = __ffs(due) - 1;
+                        due &= due - 1;
+                        uint32_t gmin = kNoFin;  // new minimum of lane c's stretch
+                        const int stop = min(nP, (c + 1) << bsh);
+                        for (int base = c << bsh; base < stop; base += 32) {
+                            const int i = base + lane;
+                            const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
+                            const bool done = (sw == (uint32_t)t);
+                            const uint32_t m = __ballot_sync(FULL, done);
+                            if (m) {
+                                if (done) {
+                                    const uint64_t e = RING(WR(head + i));
+                                    const int l = entry_l(e), o = entry_o(e);
+                                    const int lat = t - entry_tarr(e) + 1;
+                                    acc_lat += (unsigned)lat;
+                                    acc_o += (unsigned)o;
+                                    sum_lo += l + o;
+                                    acc_maxlat = max(acc_maxlat, lat);
+                                    acc_w += (unsigned long long)l * o + (unsigned long long)o * (o + 1) / 2;
+                                    if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
+                                    if (lrow) {
+                                        const int li = n_logged + ndone + __popc(m & lt_mask);  // activation order
+                                        if (li < p.complog_cap) LROW(li) = make_int2(t, lat);
+                                    }
+                                    STATE(WA(shead + i)) = kDead;
                                 }
-                                STATE(WA(shead + i)) = kDead;
+                                ndone += __popc(m);
                             }
-                            ndone += __popc(m);
+                            gmin = min(gmin, __reduce_min_sync(FULL, (done || sw == kDead) ? kNoFin : sw));
                         }
-                        const uint32_t cand = (done || sw == kDead) ? kNoFin : sw;
-                        newmin = min(newmin, cand);
+                        if (lane == c) cmin = gmin;
                     }
-                    next_fin = __reduce_min_sync(FULL, newmin);
+                    next_fin = __reduce_min_sync(FULL, cmin);
                     if (ndone > 0) {
                         nD += ndone;
                         Ndec -= ndone;
+                        completed += ndone;
                         U -= __reduce_add_sync(FULL, sum_lo);
-                        CADD(C_COMPLETED, ndone);
-                        CADD(C_SUM_LAT, __reduce_add_sync(FULL, sum_lat));
-                        CADD(C_COMPLETED_TOKENS, __reduce_add_sync(FULL, sum_o));
-                        CMAX(C_MAX_LAT, __reduce_max_sync(FULL, max_lat));
-                        CADD(C_SUM_W_COMPLETED, warp_sum64(sum_w));
                         if (lrow) {
                             if (n_logged + ndone > p.complog_cap) status |= 2u;
                             n_logged = min(p.complog_cap, n_logged + ndone);
@@ -605,6 +634,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
         CADD(C_TOKENS_GENERATED, tokgen);
         CADD(C_ARRIVED, arrived);
         CADD(C_DROPPED, dropped);
+        CADD(C_COMPLETED, completed);
+        CADD(C_SUM_LAT, warp_sum64((long long)acc_lat));
+        CADD(C_SUM_W_COMPLETED, warp_sum64((long long)acc_w));
+        CADD(C_COMPLETED_TOKENS, warp_sum64((long long)acc_o));
+        CMAX(C_MAX_LAT, __reduce_max_sync(FULL, acc_maxlat));
         CMAX(C_MAX_U, maxU);
         CMAX(C_MAX_Q, maxQ);
         CSET(C_STEPS_DONE, t_end);

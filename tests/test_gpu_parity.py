@@ -121,3 +121,20 @@ def test_host_buffer_entry_point():
     ref = orc.run(cfg)
     assert_same(cfg, out, ref, 500, "simulate_host")
     assert_summary_close(cfg, out["summary"], ref["counters"], ref["hist"], 500)
+
+
+def test_large_active_set_and_lazy_removal_paths():
+    # Acap > 1024 (several 32-entry blocks per watching lane), completions piling up between removals,
+    # removal forced by storage (active range full of completed entries) and by evictions
+    many = degenerate_config(n=40, l=1, o=3, policy="greedy", b=0, K=0, c=0, M=100000, T=120, Qcap=2000, Acap=1500)
+    many = many.with_(arrivals=(wl.Arrivals((wl.poisson_table(30.0),)),), decode=(wl.uniform_table(1, 60),),
+                      complog_cap=8192)
+    assert_same(many, run_gpu(many), orc.run(many), 120, "Acap 1500")
+    tight = wl.config1(replicas=6, T=1500).with_(
+        Acap=40, Qcap=30, M=12000, arrivals=(wl.Arrivals((wl.poisson_table(1.5),)),),
+        groups=(wl.Group(wl.POLICY_FLOW, b_fp=0x30000, n_replicas=6),))
+    ref = orc.run(tight)
+    assert ref["counters"][:, orc.CIDX["acap_blocked_steps"]].sum() > 0
+    assert_same(tight, run_gpu(tight), ref, 1500, "storage-bound")
+    churn = wl.config2(replicas=2, T=3000).with_(M=20000, Acap=96)
+    assert_same(churn, run_gpu(churn, pieces=[1000, 1, 1999]), orc.run(churn), 3000, "eviction churn")
