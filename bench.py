@@ -31,9 +31,9 @@ UNIT = "replica-steps/s"
 # Executed warp-instructions per replica-step of the step kernel in the timed regime of each preset,
 # from the committed ncu captures (profiles/): smsp__inst_executed.sum / (replicas x slots) of one launch.
 # None = not captured for the current kernel.
-INST_PER_REPLICA_STEP = {1: None, 2: None, 3: None, 4: None, 5: 343.6}
+INST_PER_REPLICA_STEP = {1: None, 2: None, 3: 344.1, 4: None, 5: 273.0}
 # DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
-DRAM_BYTES_PER_REPLICA_STEP = {1: None, 2: None, 3: None, 4: None, 5: 7.9}
+DRAM_BYTES_PER_REPLICA_STEP = {1: None, 2: None, 3: 17.9, 4: None, 5: 7.9}
 
 DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000}
 NAMES = {1: "cfg1-tiny-flow", 2: "cfg2-policy-comparison", 3: "cfg3-stability-sweep", 4: "cfg4-heavy-tail",
