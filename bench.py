@@ -31,13 +31,13 @@ UNIT = "replica-steps/s"
 # Executed warp-instructions per replica-step of the step kernel in the timed regime of each preset,
 # from the committed ncu captures (profiles/): smsp__inst_executed.sum / (replicas x slots) of one launch.
 # None = not captured for the current kernel.
-INST_PER_REPLICA_STEP = {1: None, 2: None, 3: 344.1, 4: None, 5: 273.0}
+INST_PER_REPLICA_STEP = {1: None, 2: None, 3: 344.1, 4: None, 5: 273.0, 6: None}
 # DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
-DRAM_BYTES_PER_REPLICA_STEP = {1: None, 2: None, 3: 17.9, 4: None, 5: 7.9}
+DRAM_BYTES_PER_REPLICA_STEP = {1: None, 2: None, 3: 17.9, 4: None, 5: 7.9, 6: None}
 
-DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000}
+DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000, 6: 500}
 NAMES = {1: "cfg1-tiny-flow", 2: "cfg2-policy-comparison", 3: "cfg3-stability-sweep", 4: "cfg4-heavy-tail",
-         5: "cfg5-large-bursty"}
+         5: "cfg5-large-bursty", 6: "cfg6-paper-section-4.1"}
 
 
 def make_config(workload: int, total_steps: int, rank: int = 0, replicas: int = 0):
@@ -180,7 +180,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--workload", type=int, default=5, choices=[1, 2, 3, 4, 5, 6])
     ap.add_argument("--chunk", type=int, default=0, help="slots per bench step (0 = preset default)")
     ap.add_argument("--replicas", type=int, default=0, help="replicas per group (0 = the preset's; profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

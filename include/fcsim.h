@@ -41,7 +41,10 @@ enum {
     FCSIM_ETOOBIG = -7 /* fcsim_stats_noalloc: the group rows exceed the library's fixed device scratch */
 };
 
-enum { FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2 };
+/* ALPHA is the alpha-protection greedy baseline of Section 4.1: prefill-first greedy admission that keeps
+ * the usage within (1 - alpha) M when a prompt (initial memory l + 1) joins, and evicts ALL active
+ * requests back to the waiting queue when the slot would overflow M. */
+enum { FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2, FCSIM_POLICY_ALPHA = 3 };
 
 /* Integer inverse-CDF table.  Support {vmin .. vmin+n-1}; cdf[k] = floor(P(X <= vmin+k) * 2^32) clamped
  * to 2^32-1, non-decreasing; cdf[n-1] is a catch-all whose value is ignored.  A 32-bit word u maps to
@@ -68,7 +71,8 @@ typedef struct {
  *       i.i.d., mean b_fp / 65536, bounded by (b_fp >> 16) + 1 (the law asked for by Theorem 3.6).
  * chunk: prefill chunk size c (CHUNKED only, >= 1).
  * rng_replica_base: generator replica id of the group's first replica (equal bases in two groups give
- *       common random numbers). */
+ *       common random numbers).
+ * m_admit: ALPHA only, the admission limit floor((1 - alpha) M) in tokens, 1 .. M. */
 typedef struct {
     int32_t policy;
     uint32_t b_fp;
@@ -76,6 +80,7 @@ typedef struct {
     int32_t arrivals_id;
     uint32_t rng_replica_base;
     int32_t n_replicas;
+    int32_t m_admit;
 } fcsim_group;
 
 /* M: KV capacity in tokens (1 .. 2^30).  K: prefill-token budget per slot, 0 = none (the paper's model).

@@ -2,7 +2,8 @@
 //
 // Plain, slow, single-threaded CPU simulator of the token-level serving model of
 // Section 2.1 driven by the flow-controlled policy of Algorithm 2 (and by the greedy
-// prefill-first and chunked-prefill baselines named in the Introduction).  It is
+// prefill-first and chunked-prefill baselines named in the Introduction, and the alpha-protection
+// greedy baseline described in Section 4.1).  It is
 // written directly from the paper, one request object at a time, with a std::deque
 // waiting queue and a std::vector active set; the KV usage U_t is re-summed from the
 // request objects every slot.  It shares no code, header or table with the CUDA
@@ -41,12 +42,13 @@ struct orc_arrivals {
     uint32_t switch_thr[2];
 };
 struct orc_group {
-    int32_t policy;  // 0 FLOW, 1 GREEDY, 2 CHUNKED
+    int32_t policy;  // 0 FLOW, 1 GREEDY, 2 CHUNKED, 3 ALPHA (alpha-protection greedy, Section 4.1)
     uint32_t b_fp;
     int32_t chunk;
     int32_t arrivals_id;
     uint32_t rng_replica_base;
     int32_t n_replicas;
+    int32_t m_admit;  // ALPHA: a new prompt is admitted only while usage stays <= m_admit = (1-alpha) M
 };
 struct orc_config {
     int32_t M, K, T_max, Qcap, Acap;
@@ -156,7 +158,8 @@ int validate(const orc_config& c) {
     }
     for (int g = 0; g < c.n_groups; ++g) {
         const orc_group& G = c.groups[g];
-        if (G.policy < 0 || G.policy > 2 || G.n_replicas < 1) return -1;
+        if (G.policy < 0 || G.policy > 3 || G.n_replicas < 1) return -1;
+        if (G.policy == 3 && (G.m_admit < 1 || G.m_admit > c.M)) return -1;
         if (G.arrivals_id < 0 || G.arrivals_id >= c.n_arrivals) return -1;
         if (G.policy == 2 && G.chunk < 1) return -1;
     }
@@ -172,8 +175,11 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
     const uint32_t key[2] = {(uint32_t)(cfg.seed & 0xffffffffu), (uint32_t)(cfg.seed >> 32)};
     const orc_arrivals& arr = cfg.arrivals[grp.arrivals_id];
     const int64_t INF = std::numeric_limits<int64_t>::max() / 4;
-    const bool flow = grp.policy == 0, chunked = grp.policy == 2;
+    const bool flow = grp.policy == 0, chunked = grp.policy == 2, alpha = grp.policy == 3;
     const int64_t M = cfg.M;
+    // alpha-protection greedy (Section 4.1): a new prompt with initial memory l+1 joins only if the usage
+    // stays within (1-alpha) M; every other policy admits up to the capacity itself
+    const int64_t admit_limit = alpha ? (int64_t)grp.m_admit : M;
 
     std::deque<Request> Q;
     std::vector<Request> P;
@@ -251,7 +257,7 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
                 if (!(cfg.K == 0 || a == 0 || g <= R)) { C[C_BUDGET_BLOCKED]++; break; }
                 need = (int64_t)h.l + 1;
             }
-            if (G + need > M) { C[C_GATE_BLOCKED]++; break; }
+            if (G + need > admit_limit) { C[C_GATE_BLOCKED]++; break; }
             Q.pop_front();
             h.p = (int32_t)g;
             h.j = 0;
@@ -271,7 +277,9 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
         // ---- E: overflow: evict last-in-first-out, refreshed, back to the queue front
         if (G > M) {
             C[C_OVERFLOW_STEPS]++;
-            while (G > M) {
+            // alpha-protection greedy evicts all active requests on overflow; the others evict
+            // last-in-first-out only until the slot fits
+            while (alpha ? !P.empty() : G > M) {
                 if (P.empty()) return -10;
                 Request r = P.back();
                 P.pop_back();

@@ -68,7 +68,8 @@ int plan(const fcsim_config* c, Layout* L) {
     long long R = 0;
     for (int g = 0; g < c->n_groups; ++g) {
         const fcsim_group& G = c->groups[g];
-        if (G.policy < 0 || G.policy > 2 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.policy < 0 || G.policy > 3 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.policy == FCSIM_POLICY_ALPHA && (G.m_admit < 1 || G.m_admit > c->M)) return FCSIM_EINVAL;
         if (G.arrivals_id < 0 || G.arrivals_id >= c->n_arrivals) return FCSIM_EINVAL;
         if (G.policy == FCSIM_POLICY_CHUNKED && G.chunk < 1) return FCSIM_EINVAL;
         R += G.n_replicas;
@@ -262,7 +263,8 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
     int first = 0;
     for (int g = 0; g < c->n_groups; ++g) {
         const fcsim_group& G = c->groups[g];
-        grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas, 0};
+        grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas,
+                           G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M};
         first += G.n_replicas;
     }
     CUDA_TRY(h, cudaMalloc(&h->d_gpool, gpool.size() * sizeof(unsigned short)));

@@ -58,7 +58,7 @@ struct DevGroup {
     uint32_t rng_base;
     int32_t first;  // index of the group's first replica
     int32_t n;
-    int32_t pad;
+    int32_t admit_limit;  // usage a new admission may reach: M, or (1-alpha) M for the alpha-protection policy
 };
 
 struct Params {
@@ -233,6 +233,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
         const uint32_t rid = grp.rng_base + (r - (unsigned)grp.first);
         const int policy = grp.policy;
         const int chunk = grp.chunk;
+        const int admit_limit = grp.admit_limit;
 
         // ------------------------------------------------------------------ load state
         unsigned char* ws = p.workspace + (size_t)r * p.ws_stride;
@@ -484,7 +485,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                             if (!(kinf || a == 0 || g <= R)) { CADD(C_BUDGET_BLOCKED, 1); break; }
                             need = l + 1;
                         }
-                        if (G + need > M) { CADD(C_GATE_BLOCKED, 1); break; }
+                        if (G + need > admit_limit) { CADD(C_GATE_BLOCKED, 1); break; }
                         uint32_t sw;
                         if (g == l) {
                             sw = (uint32_t)(t + entry_o(RING(WR(head + nP))) - 1);
@@ -514,7 +515,29 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                 if (G > M) {
                     CADD(C_OVERFLOW_STEPS, 1);
                     int nev = 0, wasted = 0;
-                    while (G > M && nP > 0) {
+                    if (policy == 3) {
+                        // alpha-protection greedy (Section 4.1): every active request goes back to the queue.
+                        // Completed entries were squeezed out above, so the whole active range is live and
+                        // simply becomes the front of the queue.
+                        for (int base = 0; base < nP; base += 32) {
+                            const int i = base + lane;
+                            if (i < nP) {
+                                const uint32_t sw = STATE(WA(shead + i));
+                                if (!(sw & kPrefillBit)) wasted += t - (int)sw + entry_o(RING(WR(head + i))) - 1;
+                            }
+                        }
+                        wasted = __reduce_add_sync(FULL, wasted);
+                        nev = nP;
+                        nQ += nP;
+                        nP = 0;
+                        Ndec = 0;
+                        n_pref = 0;
+                        G = 0;
+                        q_l = -1;
+                        cmin = kNoFin;
+                        next_fin = kNoFin;
+                    }
+                    while (policy != 3 && G > M && nP > 0) {
                         const int i = nP - 1;
                         const uint32_t sw = STATE(WA(shead + i));
                         const uint64_t e = RING(WR(head + i));

@@ -7,17 +7,18 @@ import numpy as np
 
 from paper_2604_11001_b200 import workloads as wl
 
-POLICIES = {"flow": wl.POLICY_FLOW, "greedy": wl.POLICY_GREEDY, "chunked": wl.POLICY_CHUNKED}
+POLICIES = {"flow": wl.POLICY_FLOW, "greedy": wl.POLICY_GREEDY, "chunked": wl.POLICY_CHUNKED,
+            "alpha": wl.POLICY_ALPHA}
 
 
-def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, **extra):
+def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, ma=0, **extra):
     """Constant arrival count n per slot, constant lengths (l, o)."""
     pol = POLICIES[policy] if isinstance(policy, str) else policy
     return wl.SimConfig(
         M=M, K=K, T_max=T, Qcap=Qcap, Acap=Acap, seed=extra.pop("seed", 7),
         class_law=wl.constant_table(0), prompt=(wl.constant_table(l),), decode=(wl.constant_table(o),),
         arrivals=(wl.Arrivals((wl.constant_table(n),)),),
-        groups=(wl.Group(pol, b_fp=wl.b_to_fp(b), chunk=c, n_replicas=replicas),),
+        groups=(wl.Group(pol, b_fp=wl.b_to_fp(b), chunk=c, n_replicas=replicas, m_admit=ma),),
         trace_stride=1, hist_bins=extra.pop("hist_bins", 16), hist_shift=0, complog_cap=4 * T, **extra)
 
 
@@ -36,7 +37,7 @@ def read_fixture(path):
         params[k] = v if k == "policy" else (float(v) if k == "b" else int(v))
     out = {"params": params, "U": [int(x) for x in fx.pop("U").split()],
            "Q": [int(x) for x in fx.pop("Q").split()],
-           "completions": [tuple(int(y) for y in x.split(":")) for x in fx.pop("completions").split()]}
+           "completions": [tuple(int(y) for y in x.split(":")) for x in fx.pop("completions", "").split()]}
     out["counters"] = {k: int(v) for k, v in fx.items()}
     return out
 
@@ -53,4 +54,5 @@ def scaled_presets():
         wl.config3(n_rates=3, n_b=3, reps=2, T=4000),
         wl.config4(replicas=3, T=4000, trace_stride=4),
         wl.config5(replicas=3, T=6000),
+        wl.config6(replicas=3, T=3000),
     ]

@@ -111,7 +111,8 @@ def brute_force(cfg, replica, n_steps):
                     cnt["budget_blocked_steps"] += 1
                     break
                 need = g + 1
-            if prospective() + need > cfg.M:
+            limit = grp.m_admit if grp.policy == 3 else cfg.M   # alpha-protection: keep usage <= (1-alpha) M
+            if prospective() + need > limit:
                 cnt["gate_blocked_steps"] += 1
                 break
             h["status"], h["p"], h["j"], h["act_seq"] = "active", g, 0, act_seq
@@ -123,7 +124,7 @@ def brute_force(cfg, replica, n_steps):
             cnt["prefill_tokens"] += g
         if prospective() > cfg.M:
             cnt["overflow_steps"] += 1
-            while prospective() > cfg.M:
+            while (active() if grp.policy == 3 else prospective() > cfg.M):   # alpha-protection evicts all
                 r = active()[-1]
                 cnt["wasted_tokens"] += r["j"]
                 cnt["evictions"] += 1

@@ -118,3 +118,12 @@ def test_config5_full():
 def test_config5_all_replicas_first_2000_slots_against_a_stratified_sample():
     cfg = wl.config5()
     _run_full(cfg, 2000, list(range(0, cfg.n_replicas, 4099)), n_steps=2000)
+
+
+def test_config6_full_paper_setting():
+    cfg = wl.config6()
+    c = _run_full(cfg, 500, _sample(cfg, 8, 6))
+    # Section 4.1's load is light (about 0.41 of the necessary-condition load): flow control with b = 12 > lambda
+    # never overflows, and nothing is dropped
+    n = cfg.groups[0].n_replicas
+    assert c[:n, I["overflow_steps"]].sum() == 0 and c[:, I["dropped"]].sum() == 0

@@ -79,3 +79,31 @@ def test_zero_flow_rate_admits_nothing_and_fractional_rate_has_the_right_mean():
     rate = out["counters"][:, I["admitted"]].sum() / (8 * 3000)
     assert abs(rate - 0.25) < 0.01
     assert out["counters"][:, I["q_final"]].min() > 100   # lambda = 0.5 > b: the queue stands
+
+
+def test_alpha_protection_with_full_limit_and_no_overflow_is_greedy():
+    # Section 4.1 baseline: with alpha = 0 the admission rule is the capacity itself; while no slot overflows
+    # the evict-all rule never fires and the policy coincides with greedy
+    cfg = wl.config6(replicas=3, T=2500)
+    n = 3
+    alpha0 = cfg.with_(groups=(wl.Group(wl.POLICY_ALPHA, n_replicas=n, m_admit=cfg.M),))
+    greedy = cfg.with_(groups=(wl.Group(wl.POLICY_GREEDY, n_replicas=n),))
+    a, g = orc.run(alpha0), orc.run(greedy)
+    assert a["counters"][:, I["overflow_steps"]].sum() == 0
+    _same(a, g)
+
+
+def test_alpha_protection_evicts_everything_on_overflow():
+    # overloaded single class: whenever a slot overflows, the active set is emptied (usage 0 in that slot)
+    cfg = wl.config1(replicas=3, T=1500)
+    cfg = cfg.with_(groups=(wl.Group(wl.POLICY_ALPHA, n_replicas=3, m_admit=cfg.M - 64),))
+    out = orc.run(cfg, admlog_cap=0)
+    c = out["counters"]
+    assert c[:, I["overflow_steps"]].min() > 0
+    # evictions per overflow slot = the whole active set, so evictions >> overflow slots
+    assert (c[:, I["evictions"]] > 3 * c[:, I["overflow_steps"]]).all()
+    zero_slots = (out["trace"][:, :, 0] == 0).sum(axis=1)
+    assert (zero_slots >= c[:, I["overflow_steps"]]).all()
+    # admission never takes the usage of an admission slot past the protection limit + growth of that slot:
+    # max_U can exceed m_admit only through decoding growth, never beyond M
+    assert (c[:, I["max_U"]] <= cfg.M).all()
