@@ -42,13 +42,15 @@ struct orc_arrivals {
     uint32_t switch_thr[2];
 };
 struct orc_group {
-    int32_t policy;  // 0 FLOW, 1 GREEDY, 2 CHUNKED, 3 ALPHA (alpha-protection greedy, Section 4.1)
+    int32_t policy;  // 0 FLOW, 1 GREEDY, 2 CHUNKED, 3 ALPHA (alpha-protection greedy, Section 4.1),
+                     // 4 CLASSFLOW (Algorithm 1: per-class budgets b_k, FIFO within a class)
     uint32_t b_fp;
     int32_t chunk;
     int32_t arrivals_id;
     uint32_t rng_replica_base;
     int32_t n_replicas;
     int32_t m_admit;  // ALPHA: a new prompt is admitted only while usage stays <= m_admit = (1-alpha) M
+    const int32_t* b_class;  // CLASSFLOW (policy 4, Algorithm 1): activation budget b_k of every class
 };
 struct orc_config {
     int32_t M, K, T_max, Qcap, Acap;
@@ -70,6 +72,7 @@ struct orc_outputs {
     int32_t* hist;       // [n][hist_bins]
     int32_t* complog;    // [n][complog_cap][2] = {t_done, latency}
     int32_t* arrlog;     // [n][n_steps]  n_t of every slot                    (diagnostic)
+    int32_t* arrcls;     // [n][n_steps][n_classes] arrivals of every class     (diagnostic)
     int32_t* admlog;     // [n][admlog_cap][4] = {slot, l, o, t_arr} per admission (diagnostic)
     int64_t admlog_cap;
     int64_t* n_admlog;   // [n]
@@ -158,7 +161,12 @@ int validate(const orc_config& c) {
     }
     for (int g = 0; g < c.n_groups; ++g) {
         const orc_group& G = c.groups[g];
-        if (G.policy < 0 || G.policy > 3 || G.n_replicas < 1) return -1;
+        if (G.policy < 0 || G.policy > 4 || G.n_replicas < 1) return -1;
+        if (G.policy == 4) {
+            if (!G.b_class) return -1;
+            for (int k = 0; k < c.n_classes; ++k)
+                if (G.b_class[k] < 0 || G.b_class[k] > 65535) return -1;
+        }
         if (G.policy == 3 && (G.m_admit < 1 || G.m_admit > c.M)) return -1;
         if (G.arrivals_id < 0 || G.arrivals_id >= c.n_arrivals) return -1;
         if (G.policy == 2 && G.chunk < 1) return -1;
@@ -170,12 +178,13 @@ int validate(const orc_config& c) {
 // One replica, slots 1..n_steps.  Returns 0, or a negative code if an invariant of the
 // model is violated (that would be a bug in this file, not a property of the inputs).
 int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replica, int32_t n_steps,
-                int64_t* C, int32_t* trace, int32_t* hist, int32_t* complog, int32_t* arrlog,
+                int64_t* C, int32_t* trace, int32_t* hist, int32_t* complog, int32_t* arrlog, int32_t* arrcls,
                 int32_t* admlog, int64_t admlog_cap, int64_t* n_admlog_out) {
     const uint32_t key[2] = {(uint32_t)(cfg.seed & 0xffffffffu), (uint32_t)(cfg.seed >> 32)};
     const orc_arrivals& arr = cfg.arrivals[grp.arrivals_id];
     const int64_t INF = std::numeric_limits<int64_t>::max() / 4;
     const bool flow = grp.policy == 0, chunked = grp.policy == 2, alpha = grp.policy == 3;
+    const bool classflow = grp.policy == 4;
     const int64_t M = cfg.M;
     // alpha-protection greedy (Section 4.1): a new prompt with initial memory l+1 joins only if the usage
     // stays within (1-alpha) M; every other policy admits up to the capacity itself
@@ -210,6 +219,7 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
             r.t_arr = t;
             r.p = 0;
             r.j = 0;
+            if (arrcls) arrcls[(int64_t)(t - 1) * cfg.n_classes + r.cls]++;
             C[C_ARRIVED]++;
             if ((int64_t)Q.size() >= (int64_t)cfg.Qcap) {
                 C[C_DROPPED]++;
@@ -243,7 +253,42 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
 
         // ---- D: activation, FIFO, at most B_t requests under flow control (Alg. 2 inner loop)
         int64_t a = 0;
-        const int64_t cap = flow ? B_t : INF;
+        const int64_t cap = classflow ? 0 : (flow ? B_t : INF);
+        if (classflow) {
+            // Algorithm 1: for every class k, activate up to b_k waiting requests of that class, first
+            // come first served within the class.  A pick that does not fit the cache (or the token
+            // budget) ends the loop of its class only; a full active-set storage ends the slot's activation.
+            bool gate_hit = false, budget_hit = false, storage_hit = false;
+            for (int32_t k = 0; k < cfg.n_classes && !storage_hit; ++k) {
+                for (int32_t ak = 0; ak < grp.b_class[k]; ++ak) {
+                    auto it = Q.begin();
+                    while (it != Q.end() && it->cls != k) ++it;
+                    if (it == Q.end()) break;
+                    if ((int64_t)P.size() == (int64_t)cfg.Acap) { storage_hit = true; break; }
+                    Request h = *it;
+                    const int64_t g = h.l, need = (int64_t)h.l + 1;
+                    if (!(cfg.K == 0 || a == 0 || g <= R)) { budget_hit = true; break; }
+                    if (G + need > M) { gate_hit = true; break; }
+                    Q.erase(it);
+                    h.p = (int32_t)g;
+                    h.j = 0;
+                    P.push_back(h);
+                    G += need;
+                    if (R != INF) R -= std::min(g, R);
+                    a++;
+                    C[C_ADMITTED]++;
+                    C[C_PREFILL_TOKENS] += g;
+                    if (admlog && n_admlog < admlog_cap) {
+                        int32_t* e = admlog + 4 * n_admlog;
+                        e[0] = t; e[1] = h.l; e[2] = h.o; e[3] = h.t_arr;
+                    }
+                    n_admlog++;
+                }
+            }
+            C[C_GATE_BLOCKED] += gate_hit;
+            C[C_BUDGET_BLOCKED] += budget_hit;
+            C[C_ACAP_BLOCKED] += storage_hit;
+        }
         while (a < cap && !Q.empty()) {
             if ((int64_t)P.size() == (int64_t)cfg.Acap) { C[C_ACAP_BLOCKED]++; break; }
             Request h = Q.front();
@@ -343,10 +388,20 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
         }
         C[C_MAX_Q] = std::max<int64_t>(C[C_MAX_Q], (int64_t)Q.size());
 
-        // active set followed by the queue must stay sorted by arrival order
-        int64_t prev = -1;
-        for (const Request& r : P) { if (r.id <= prev) return -13; prev = r.id; }
-        for (const Request& r : Q) { if (r.id <= prev) return -13; prev = r.id; }
+        if (!classflow) {
+            // active set followed by the queue must stay sorted by arrival order
+            int64_t prev = -1;
+            for (const Request& r : P) { if (r.id <= prev) return -13; prev = r.id; }
+            for (const Request& r : Q) { if (r.id <= prev) return -13; prev = r.id; }
+        } else {
+            // per class: active requests are older than waiting ones, and the queue is in arrival order
+            std::vector<int64_t> newest_active(cfg.n_classes, -1), prev(cfg.n_classes, -1);
+            for (const Request& r : P) newest_active[r.cls] = std::max(newest_active[r.cls], r.id);
+            for (const Request& r : Q) {
+                if (r.id <= prev[r.cls] || r.id <= newest_active[r.cls]) return -13;
+                prev[r.cls] = r.id;
+            }
+        }
     }
 
     C[C_STEPS_DONE] = n_steps;
@@ -392,6 +447,7 @@ extern "C" int fcsim_oracle_run(const orc_config* cfg, int64_t first_replica, in
         int rc = run_replica(*cfg, grp, rng_replica, n_steps, out->counters + k * C_COUNT,
                              (out->trace && n_rec > 0) ? out->trace + 2 * k * n_rec : nullptr, hist, complog,
                              out->arrlog ? out->arrlog + k * (int64_t)n_steps : nullptr,
+                             out->arrcls ? out->arrcls + k * (int64_t)n_steps * cfg->n_classes : nullptr,
                              out->admlog ? out->admlog + 4 * k * out->admlog_cap : nullptr, out->admlog_cap,
                              out->n_admlog ? out->n_admlog + k : nullptr);
         if (rc) return rc;

@@ -39,7 +39,7 @@ class _Arrivals(C.Structure):
 class _Group(C.Structure):
     _fields_ = [("policy", C.c_int32), ("b_fp", C.c_uint32), ("chunk", C.c_int32),
                 ("arrivals_id", C.c_int32), ("rng_replica_base", C.c_uint32), ("n_replicas", C.c_int32),
-                ("m_admit", C.c_int32)]
+                ("m_admit", C.c_int32), ("b_class", C.POINTER(C.c_int32))]
 
 
 class _Config(C.Structure):
@@ -55,7 +55,8 @@ class _Config(C.Structure):
 class _Outputs(C.Structure):
     _fields_ = [("counters", C.POINTER(C.c_int64)), ("trace", C.POINTER(C.c_int32)),
                 ("hist", C.POINTER(C.c_int32)), ("complog", C.POINTER(C.c_int32)),
-                ("arrlog", C.POINTER(C.c_int32)), ("admlog", C.POINTER(C.c_int32)),
+                ("arrlog", C.POINTER(C.c_int32)), ("arrcls", C.POINTER(C.c_int32)),
+                ("admlog", C.POINTER(C.c_int32)),
                 ("admlog_cap", C.c_int64), ("n_admlog", C.POINTER(C.c_int64))]
 
 
@@ -101,8 +102,14 @@ def marshal(cfg):
         arrs[i].switch_thr[1] = int(a.switch_thr[1])
     groups = (_Group * len(cfg.groups))()
     for i, g in enumerate(cfg.groups):
+        bc = getattr(g, "b_class", ())
+        bptr = None
+        if len(bc):
+            arr = np.ascontiguousarray(bc, dtype=np.int32)
+            keep.append(arr)
+            bptr = arr.ctypes.data_as(C.POINTER(C.c_int32))
         groups[i] = _Group(int(g.policy), int(g.b_fp), int(g.chunk), int(g.arrivals_id),
-                           int(g.rng_replica_base), int(g.n_replicas), int(getattr(g, "m_admit", 0)))
+                           int(g.rng_replica_base), int(g.n_replicas), int(getattr(g, "m_admit", 0)), bptr)
     c = _Config(int(cfg.M), int(cfg.K), int(cfg.T_max), int(cfg.Qcap), int(cfg.Acap), int(cfg.seed),
                 len(cfg.prompt), _mk_table(cfg.class_law, keep), prompt, decode, len(cfg.arrivals), arrs,
                 len(cfg.groups), groups, int(cfg.trace_stride), int(cfg.hist_bins), int(cfg.hist_shift),
@@ -129,7 +136,7 @@ def _p(arr, typ):
     return arr.ctypes.data_as(C.POINTER(typ)) if arr is not None else None
 
 
-def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize):
+def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize, arrcls=False):
     c, keep = marshal(cfg)
     out = {"counters": np.zeros((n, N_COUNTERS), dtype=np.int64)}
     n_rec = n_steps // cfg.trace_stride if cfg.trace_stride > 0 else 0
@@ -138,10 +145,12 @@ def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap,
     out["complog"] = (np.zeros((n, cfg.complog_cap, 2), dtype=np.int32)
                       if (complog and cfg.complog_cap > 0) else None)
     out["arrlog"] = np.zeros((n, n_steps), dtype=np.int32) if arrlog else None
+    out["arrcls"] = np.zeros((n, n_steps, len(cfg.prompt)), dtype=np.int32) if arrcls else None
     out["admlog"] = np.zeros((n, admlog_cap, 4), dtype=np.int32) if admlog_cap > 0 else None
     out["n_admlog"] = np.zeros(n, dtype=np.int64) if admlog_cap > 0 else None
     o = _Outputs(_p(out["counters"], C.c_int64), _p(out["trace"], C.c_int32), _p(out["hist"], C.c_int32),
-                 _p(out["complog"], C.c_int32), _p(out["arrlog"], C.c_int32), _p(out["admlog"], C.c_int32),
+                 _p(out["complog"], C.c_int32), _p(out["arrlog"], C.c_int32), _p(out["arrcls"], C.c_int32),
+                 _p(out["admlog"], C.c_int32),
                  int(admlog_cap), _p(out["n_admlog"], C.c_int64))
     rc = lib(sanitize).fcsim_oracle_run(C.byref(c), int(first), int(n), int(n_steps), C.byref(o))
     if rc != 0:
@@ -151,7 +160,7 @@ def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap,
 
 
 def run(cfg, first_replica=0, n_replicas=None, n_steps=None, *, trace=True, hist=True, complog=True,
-        arrlog=False, admlog_cap=0, threads=1, sanitize=False):
+        arrlog=False, admlog_cap=0, threads=1, sanitize=False, arrcls=False):
     """Simulate replicas [first_replica, first_replica+n_replicas) for slots 1..n_steps.
 
     Returns a dict of numpy arrays: counters [n,28] int64, and (when enabled in ``cfg`` and
@@ -166,11 +175,11 @@ def run(cfg, first_replica=0, n_replicas=None, n_steps=None, *, trace=True, hist
     threads = max(1, min(int(threads), n_replicas)) if n_replicas > 0 else 1
     if threads == 1:
         return _run_range(cfg, first_replica, n_replicas, n_steps, trace, hist, complog, arrlog,
-                          admlog_cap, sanitize)
+                          admlog_cap, sanitize, arrcls)
     bounds = np.linspace(0, n_replicas, threads + 1).astype(np.int64)
     with ThreadPoolExecutor(max_workers=threads) as ex:
         futs = [ex.submit(_run_range, cfg, first_replica + int(bounds[i]), int(bounds[i + 1] - bounds[i]),
-                          n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize)
+                          n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize, arrcls)
                 for i in range(threads)]
         parts = [f.result() for f in futs]
     out = {}

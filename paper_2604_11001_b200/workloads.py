@@ -30,6 +30,7 @@ POLICY_FLOW = 0
 POLICY_GREEDY = 1
 POLICY_CHUNKED = 2
 POLICY_ALPHA = 3   # alpha-protection greedy (Section 4.1)
+POLICY_CLASSFLOW = 4   # Algorithm 1: per-class activation budgets b_k, FIFO within a class
 
 _TWO32 = float(2 ** 32)
 
@@ -163,6 +164,7 @@ class Group:
     rng_replica_base: int = 0  # generator replica id = base + index within the group
     n_replicas: int = 1
     m_admit: int = 0           # ALPHA: admission keeps usage <= m_admit = floor((1 - alpha) M)
+    b_class: Tuple[int, ...] = ()  # CLASSFLOW: integer budget b_k of every class (Algorithm 1)
 
 
 @dataclass(frozen=True)
@@ -321,7 +323,8 @@ def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2) -> SimConf
     """The paper's own synthetic setting (Section 4.1): three classes (l, o) = (10,20), (10,40), (10,60),
     Poisson arrivals of total intensity 5 per slot split evenly over the classes, M = 16492, no token
     budget, T up to 10000.  Policies on common random numbers: Algorithm 2 with b = 12 (the sum of the
-    paper's per-class budgets 4+4+4), greedy, and alpha-protection greedy."""
+    paper's per-class budgets 4+4+4), greedy, alpha-protection greedy, and Algorithm 1 with the paper's
+    budgets (4, 4, 4), for which sum_k b_k w_k = 16240 < M (Eq. 2)."""
     class_law = Table(0, np.array([1431655765, 2863311530, 0xFFFFFFFF], dtype=np.uint32))
     prompt = tuple(constant_table(10) for _ in range(3))
     decode = tuple(constant_table(o) for o in (20, 40, 60))
@@ -331,7 +334,8 @@ def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2) -> SimConf
         arrivals=(Arrivals((poisson_table(5.0),)),),
         groups=(Group(POLICY_FLOW, b_fp=12 << 16, n_replicas=replicas),
                 Group(POLICY_GREEDY, n_replicas=replicas),
-                Group(POLICY_ALPHA, n_replicas=replicas, m_admit=int(math.floor((1.0 - alpha) * M)))),
+                Group(POLICY_ALPHA, n_replicas=replicas, m_admit=int(math.floor((1.0 - alpha) * M))),
+                Group(POLICY_CLASSFLOW, n_replicas=replicas, b_class=(4, 4, 4))),
         trace_stride=1, hist_bins=1024, hist_shift=0, complog_cap=0, name="cfg6-paper-section-4.1")
 
 
@@ -365,10 +369,11 @@ def random_small_config(seed: int, n_replicas: int = 4, T: int = 60) -> SimConfi
                                      (int(rng.integers(0, 2 ** 31)), int(rng.integers(0, 2 ** 31)))))
     groups = []
     base = 0
-    for pol in (POLICY_FLOW, POLICY_GREEDY, POLICY_CHUNKED, POLICY_ALPHA):
+    for pol in (POLICY_FLOW, POLICY_GREEDY, POLICY_CHUNKED, POLICY_ALPHA, POLICY_CLASSFLOW):
         groups.append(Group(pol, b_fp=int(rng.integers(0, 3 * 65536)), chunk=int(rng.integers(1, 9)),
                             arrivals_id=int(rng.integers(0, 2)), rng_replica_base=base,
-                            n_replicas=n_replicas, m_admit=int(rng.integers(max(2, M // 2), M + 1))))
+                            n_replicas=n_replicas, m_admit=int(rng.integers(max(2, M // 2), M + 1)),
+                            b_class=tuple(int(x) for x in rng.integers(0, 3, size=n_classes))))
         base += int(rng.integers(0, 2)) * n_replicas
     stride = int(rng.choice([1, 1, 2, 3]))
     return SimConfig(

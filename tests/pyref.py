@@ -77,7 +77,7 @@ def brute_force(cfg, replica, n_steps):
             if len(waiting()) >= cfg.Qcap:
                 cnt["dropped"] += 1
             else:
-                reqs.append(dict(id=len(reqs), l=l, o=o, t_arr=t, status="wait", act_seq=None, p=0, j=0))
+                reqs.append(dict(id=len(reqs), cls=cls, l=l, o=o, t_arr=t, status="wait", act_seq=None, p=0, j=0))
         n_dec_start = sum(1 for r in active() if r["p"] == r["l"])
         room = None if cfg.K == 0 else (max(0, cfg.K - n_dec_start) if grp.policy == 2 else cfg.K)
         if grp.policy == 2:
@@ -89,7 +89,38 @@ def brute_force(cfg, replica, n_steps):
                         room -= g
                     cnt["prefill_tokens"] += g
         admitted_now = 0
-        while True:
+        if grp.policy == 4:
+            # Algorithm 1: per class k up to b_k picks, oldest waiting request of that class first
+            hits = set()
+            stop = False
+            for k in range(len(cfg.prompt)):
+                if stop:
+                    break
+                for _ in range(grp.b_class[k]):
+                    cand = [r for r in waiting() if r["cls"] == k]
+                    if not cand:
+                        break
+                    if len(active()) == cfg.Acap:
+                        hits.add("acap_blocked_steps")
+                        stop = True
+                        break
+                    h = cand[0]
+                    if not (room is None or admitted_now == 0 or h["l"] <= room):
+                        hits.add("budget_blocked_steps")
+                        break
+                    if prospective() + h["l"] + 1 > cfg.M:
+                        hits.add("gate_blocked_steps")
+                        break
+                    h["status"], h["p"], h["j"], h["act_seq"] = "active", h["l"], 0, act_seq
+                    act_seq += 1
+                    if room is not None:
+                        room -= min(h["l"], room)
+                    admitted_now += 1
+                    cnt["admitted"] += 1
+                    cnt["prefill_tokens"] += h["l"]
+            for name in hits:
+                cnt[name] += 1
+        while grp.policy != 4:
             if grp.policy == 0 and admitted_now >= B_t:
                 break
             wq = waiting()

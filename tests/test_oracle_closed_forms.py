@@ -96,3 +96,59 @@ def test_percentile_rule_and_summaries():
     assert s["mean_utilisation"] == sum((3, 7, 9, 8, 7, 9, 8, 7, 9, 8, 7, 9)) / (12 * 11)
     # token throughput: tokens generated per slot (Section 2.2)
     assert s["token_throughput"] == out["counters"][0, I["tokens_generated"]] / 12
+
+
+# ---------------------------------------------------------------- Algorithm 1 (per-class budgets, known lengths)
+def _paper_classes(T, lam, b=(4, 4, 4), M=16492, replicas=3, Qcap=2 ** 31 - 1):
+    cfg = wl.config6(replicas=replicas, T=T)
+    return cfg.with_(M=M, Qcap=Qcap, Acap=4096, arrivals=(wl.Arrivals((wl.poisson_table(lam),)),),
+                     groups=(wl.Group(wl.POLICY_CLASSFLOW, n_replicas=replicas, b_class=tuple(b)),))
+
+
+def test_algorithm1_section_4_1_never_exceeds_the_bound_of_theorem_3_3():
+    # Section 4.1: (l,o) = (10,20),(10,40),(10,60), b = (4,4,4): usage <= sum_k b_k w_k = 16240 < M = 16492
+    # in every slot, so no eviction ever happens and the gate never binds (proof of Thm. 3.3)
+    cfg = _paper_classes(T=6000, lam=5.0)
+    out = orc.run(cfg)
+    c = out["counters"]
+    assert (c[:, I["max_U"]] <= 16240).all()
+    assert c[:, I["evictions"]].sum() == 0 and c[:, I["gate_blocked_steps"]].sum() == 0
+    assert c[:, I["completed"]].min() > 25000
+    # integer b_k > lambda_k = 5/3: queues are positive recurrent -- short and bounded
+    assert c[:, I["max_Q"]].max() < 40
+
+
+def test_algorithm1_saturated_usage_equals_sum_b_k_w_k():
+    # with at least b_k waiting requests of every class in every slot the bound is attained exactly
+    cfg = _paper_classes(T=400, lam=60.0)
+    out = orc.run(cfg, complog=False, hist=False)
+    assert (out["trace"][:, 80:, 0] == 16240).all()
+    assert (out["trace"][:, :59, 0] < 16240).all()
+
+
+def test_algorithm1_per_class_queues_follow_the_lindley_recursion():
+    # proof of Thm. 3.3: Q_{t,k} = (Q_{t-1,k} + n_{t,k} - b_k)^+, independently for every class
+    cfg = _paper_classes(T=3000, lam=5.5, b=(2, 2, 1), M=2 ** 30)
+    out = orc.run(cfg, arrcls=True, complog=False, hist=False)
+    assert out["counters"][:, I["evictions"]].sum() == 0
+    for r in range(cfg.n_replicas):
+        q = np.zeros(3, dtype=np.int64)
+        expect = []
+        for n_tk in out["arrcls"][r]:
+            q = np.maximum(q + n_tk - np.array([2, 2, 1]), 0)
+            expect.append(int(q.sum()))
+        assert out["trace"][r, :, 1].tolist() == expect
+        assert (out["arrcls"][r].sum(axis=1) >= 0).all()
+    # class 3 has b_3 = 1 < lambda_3: its queue grows, the others stay short
+    assert out["trace"][:, -1, 1].min() > 1000
+
+
+def test_algorithm1_with_one_class_is_algorithm2_with_integer_budget():
+    base = wl.config1(replicas=4, T=1500)
+    for b in (1, 2):
+        one = base.with_(groups=(wl.Group(wl.POLICY_CLASSFLOW, n_replicas=4, b_class=(b,)),))
+        flow = base.with_(groups=(wl.Group(wl.POLICY_FLOW, b_fp=b << 16, n_replicas=4),))
+        a, f = orc.run(one), orc.run(flow)
+        for k in ("trace", "hist", "complog"):
+            assert (a[k] == f[k]).all()
+        assert (a["counters"] == f["counters"]).all()
