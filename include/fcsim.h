@@ -44,7 +44,14 @@ enum {
 /* ALPHA is the alpha-protection greedy baseline of Section 4.1: prefill-first greedy admission that keeps
  * the usage within (1 - alpha) M when a prompt (initial memory l + 1) joins, and evicts ALL active
  * requests back to the waiting queue when the slot would overflow M. */
-enum { FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2, FCSIM_POLICY_ALPHA = 3 };
+/* CLASSFLOW is Algorithm 1 (known output length): every slot, for each class k in turn, up to b_k waiting
+ * requests of that class are activated, first come first served within the class.  The memory gate, the
+ * token budget and the last-in-first-out eviction are those of Algorithm 2 (they never act when the
+ * condition of Theorem 3.3 holds); a pick that does not fit ends the loop of its class only. */
+enum {
+    FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2, FCSIM_POLICY_ALPHA = 3,
+    FCSIM_POLICY_CLASSFLOW = 4
+};
 
 /* Integer inverse-CDF table.  Support {vmin .. vmin+n-1}; cdf[k] = floor(P(X <= vmin+k) * 2^32) clamped
  * to 2^32-1, non-decreasing; cdf[n-1] is a catch-all whose value is ignored.  A 32-bit word u maps to
@@ -72,7 +79,9 @@ typedef struct {
  * chunk: prefill chunk size c (CHUNKED only, >= 1).
  * rng_replica_base: generator replica id of the group's first replica (equal bases in two groups give
  *       common random numbers).
- * m_admit: ALPHA only, the admission limit floor((1 - alpha) M) in tokens, 1 .. M. */
+ * m_admit: ALPHA only, the admission limit floor((1 - alpha) M) in tokens, 1 .. M.
+ * b_class: CLASSFLOW only, HOST array [n_classes] of the integer budgets b_k (0 .. 65535), borrowed during
+ *       fcsim_create / fcsim_query_sizes; NULL otherwise. */
 typedef struct {
     int32_t policy;
     uint32_t b_fp;
@@ -81,6 +90,7 @@ typedef struct {
     uint32_t rng_replica_base;
     int32_t n_replicas;
     int32_t m_admit;
+    const int32_t* b_class;
 } fcsim_group;
 
 /* M: KV capacity in tokens (1 .. 2^30).  K: prefill-token budget per slot, 0 = none (the paper's model).

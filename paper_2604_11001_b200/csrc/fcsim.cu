@@ -23,7 +23,7 @@ constexpr int kStatsChunk = 256;             // replicas reduced by one block be
 
 struct Layout {
     int RC, Apad, S;
-    size_t ws_stride, smem_per_warp;
+    size_t ws_stride, smem_per_warp, qcnt_off;  // qcnt_off: per-class queue counts (Algorithm 1), 0 = unused
     int warps_per_block;
     int n_rec;
     long long R;
@@ -66,9 +66,16 @@ int plan(const fcsim_config* c, Layout* L) {
         }
     }
     long long R = 0;
+    bool any_classflow = false;
     for (int g = 0; g < c->n_groups; ++g) {
         const fcsim_group& G = c->groups[g];
-        if (G.policy < 0 || G.policy > 3 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.policy < 0 || G.policy > 4 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.policy == FCSIM_POLICY_CLASSFLOW) {
+            if (!G.b_class) return FCSIM_EINVAL;
+            for (int k = 0; k < c->n_classes; ++k)
+                if (G.b_class[k] < 0 || G.b_class[k] > 65535) return FCSIM_EINVAL;
+            any_classflow = true;
+        }
         if (G.policy == FCSIM_POLICY_ALPHA && (G.m_admit < 1 || G.m_admit > c->M)) return FCSIM_EINVAL;
         if (G.arrivals_id < 0 || G.arrivals_id >= c->n_arrivals) return FCSIM_EINVAL;
         if (G.policy == FCSIM_POLICY_CHUNKED && G.chunk < 1) return FCSIM_EINVAL;
@@ -84,7 +91,9 @@ int plan(const fcsim_config* c, Layout* L) {
     L->Apad = (int)align_up((size_t)c->Acap, 4);
     L->S = (int)align_up((size_t)std::max(128, max_count), 2);
     L->ws_stride = kHeaderWords * 4 + (size_t)L->RC * 8 + (size_t)L->Apad * 4;
-    L->smem_per_warp = (size_t)L->RC * 8 + (size_t)L->Apad * 4 + (size_t)L->S * 8;
+    L->qcnt_off = (size_t)L->RC * 8 + (size_t)L->Apad * 4 + (size_t)L->S * 8;
+    L->smem_per_warp = L->qcnt_off + (any_classflow ? align_up((size_t)c->n_classes * 4, 16) : 0);
+    if (!any_classflow) L->qcnt_off = 0;
     if (L->smem_per_warp > kSmemBudget) return FCSIM_ECAP;
     int w = kWarpsPerBlock;
     while (w > 1 && (size_t)w * L->smem_per_warp > kSmemBudget) w >>= 1;
@@ -191,6 +200,8 @@ struct fcsim {
     Params params;
     uint32_t* d_pool = nullptr;
     unsigned short* d_gpool = nullptr;
+    int32_t* d_bclass = nullptr;
+    void (*kernel)(const Params) = nullptr;  // step kernel variant for this configuration
     DevTable* d_tables = nullptr;
     DevArrivals* d_arrivals = nullptr;
     DevGroup* d_groups = nullptr;
@@ -260,13 +271,21 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         arrs[a].thr[1] = A.switch_thr[1];
     }
     std::vector<DevGroup> grps(c->n_groups);
+    std::vector<int32_t> bclass(1, 0);
     int first = 0;
     for (int g = 0; g < c->n_groups; ++g) {
         const fcsim_group& G = c->groups[g];
+        int32_t boff = 0;
+        if (G.policy == FCSIM_POLICY_CLASSFLOW) {
+            boff = (int32_t)bclass.size();
+            bclass.insert(bclass.end(), G.b_class, G.b_class + c->n_classes);
+        }
         grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas,
-                           G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M};
+                           G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M, boff, 0};
         first += G.n_replicas;
     }
+    CUDA_TRY(h, cudaMalloc(&h->d_bclass, bclass.size() * sizeof(int32_t)));
+    CUDA_TRY(h, cudaMemcpy(h->d_bclass, bclass.data(), bclass.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
     CUDA_TRY(h, cudaMalloc(&h->d_gpool, gpool.size() * sizeof(unsigned short)));
     CUDA_TRY(h, cudaMemcpy(h->d_gpool, gpool.data(), gpool.size() * sizeof(unsigned short), cudaMemcpyHostToDevice));
     CUDA_TRY(h, cudaMalloc(&h->d_pool, pool.size() * sizeof(uint32_t)));
@@ -288,6 +307,7 @@ static void release(fcsim* h) {
     if (!h) return;
     cudaFree(h->d_pool);
     cudaFree(h->d_gpool);
+    cudaFree(h->d_bclass);
     cudaFree(h->d_tables);
     cudaFree(h->d_arrivals);
     cudaFree(h->d_groups);
@@ -340,10 +360,11 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
 
     const size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
     if (smem_block > (size_t)prop.sharedMemPerBlockOptin) return fail(FCSIM_ECAP);
-    e = cudaFuncSetAttribute(fcsim_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block);
+    h->kernel = L.qcnt_off ? fcsim_step_kernel<true> : fcsim_step_kernel<false>;
+    e = cudaFuncSetAttribute(h->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block);
     if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
     int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fcsim_step_kernel, L.warps_per_block * 32, smem_block);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, h->kernel, L.warps_per_block * 32, smem_block);
     if (e != cudaSuccess || occ < 1) { h->last_cuda = (int)e; return fail(e != cudaSuccess ? FCSIM_ECUDA : FCSIM_ECAP); }
     h->blocks_per_sm = occ;
     const long long want = (L.R + L.warps_per_block - 1) / L.warps_per_block;
@@ -372,6 +393,8 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.trace_stride = cfg->trace_stride; p.n_rec = L.n_rec;
     p.hist_bins = cfg->hist_bins; p.hist_shift = cfg->hist_shift; p.complog_cap = cfg->complog_cap;
     p.gpool = h->d_gpool;
+    p.bclass = h->d_bclass;
+    p.qcnt_off = (uint32_t)L.qcnt_off;
     p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
     p.workspace = static_cast<unsigned char*>(b->workspace);
     p.ws_stride = L.ws_stride;
@@ -405,7 +428,7 @@ extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
         p.t0 = h->t_done;
         p.n_steps = now;
         CUDA_TRY(h, cudaMemsetAsync(h->d_work, 0, sizeof(unsigned int), st));
-        fcsim_step_kernel<<<h->grid, h->L.warps_per_block * 32, smem_block, st>>>(p);
+        h->kernel<<<h->grid, h->L.warps_per_block * 32, smem_block, st>>>(p);
         CUDA_TRY(h, cudaGetLastError());
         h->t_done += now;
         left -= now;

@@ -59,6 +59,8 @@ struct DevGroup {
     int32_t first;  // index of the group's first replica
     int32_t n;
     int32_t admit_limit;  // usage a new admission may reach: M, or (1-alpha) M for the alpha-protection policy
+    int32_t bclass_off;   // Algorithm 1: index of the group's per-class budgets in Params::bclass
+    int32_t pad;
 };
 
 struct Params {
@@ -69,6 +71,8 @@ struct Params {
     int32_t t0, n_steps;
     const uint32_t* pool;         // all thresholds
     const unsigned short* gpool;  // guide tables: for bucket b of the top bits of u, the first candidate index
+    const int32_t* bclass;        // per-class budgets b_k of the Algorithm-1 groups
+    uint32_t qcnt_off;            // byte offset of the per-class queue counts in a warp's shared memory (0 = none)
     const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
     const DevArrivals* arrivals;
     const DevGroup* groups;
@@ -153,6 +157,7 @@ __device__ __forceinline__ uint64_t pack_entry(int l, int o, int t_arr, int cls)
 __device__ __forceinline__ int entry_l(uint64_t e) { return (int)((uint32_t)e & 0xffffu); }
 __device__ __forceinline__ int entry_o(uint64_t e) { return (int)((uint32_t)e >> 16); }
 __device__ __forceinline__ int entry_tarr(uint64_t e) { return (int)((uint32_t)(e >> 32) & 0xffffffu); }
+__device__ __forceinline__ int entry_cls(uint64_t e) { return (int)(e >> 56); }
 
 // Index-checked build (-DFCSIM_CHECKED): every shared-memory and output index is compared with its
 // bound; a bad one is recorded (line, index, bound, replica) in Params::debug and the access goes to a
@@ -190,6 +195,9 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define FCSIM_MIN_CTAS 5
 #endif
 
+// kClassFlow: compiled with the per-class activation of Algorithm 1 (policy 4); the variant without it is
+// used when no group asks for it, so that the common policies do not carry its code.
+template <bool kClassFlow>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_step_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
@@ -199,6 +207,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
     uint32_t* state = reinterpret_cast<uint32_t*>(my + (size_t)p.RC * 8);
     uint64_t* stage = reinterpret_cast<uint64_t*>(my + (size_t)p.RC * 8 + (size_t)p.Apad * 4);
     const int state_bytes = p.RC * 8 + p.Apad * 4;  // multiple of 16 (host guarantees)
+    uint32_t* qcnt = reinterpret_cast<uint32_t*>(my + p.qcnt_off);  // waiting requests per class (Algorithm 1 only)
 
     const int RC = p.RC, Acap = p.Acap, Qcap = p.Qcap, M = p.M, K = p.K, S = p.S;
     const bool kinf = (K == 0);
@@ -335,6 +344,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
             next_fin = __reduce_min_sync(FULL, cmin);
         };
         rebuild_minima();
+        if ((kClassFlow && policy == 4)) {  // Algorithm 1 picks per class: count the waiting requests of every class
+            for (int c = lane; c < p.n_classes; c += 32) qcnt[c] = 0;
+            __syncwarp();
+            for (int i = lane; i < nQ; i += 32) atomicAdd(&qcnt[entry_cls(RING(WR(head + nP + i)))], 1u);
+            __syncwarp();
+        }
 
         while (t < t_end) {
             // -------------------------------------------------------------- batch: draws of up to 32 slots
@@ -404,7 +419,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                     const int acc = min(n_t, max(0, Qcap - nQ));
                     if (acc > 0) {
                         const int tail = WR(head + nP + nQ);
-                        for (int i = lane; i < acc; i += 32) RING(WR(tail + i)) = STAGE(sp + i);
+                        for (int i = lane; i < acc; i += 32) {
+                            const uint64_t e = STAGE(sp + i);
+                            RING(WR(tail + i)) = e;
+                            if ((kClassFlow && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
+                        }
                         nQ += acc;
                         __syncwarp();
                     }
@@ -461,13 +480,73 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
 
                 // ---- completed entries must be gone before an eviction (the newest entry has to be a live
                 //      one), before the active range runs out of storage, and when too many have piled up
-                bool squeeze = nD > 0 && (nD >= kCompactAt || G > M);
+                bool squeeze = nD > 0 && (nD >= kCompactAt || G > M || ((kClassFlow && policy == 4) && nP + nQ > Acap));
 
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
                 int a = 0;
                 const int cap = (policy == 0) ? B_t : 0x7fffffff;
                 for (;;) {
                     if (squeeze) { compact(); rebuild_minima(); squeeze = false; }
+                    if ((kClassFlow && policy == 4)) {
+                        // Algorithm 1: for every class k, up to b_k waiting requests of that class, oldest first.
+                        // The pick leaves the middle of the queue: the entries ahead of it move one place
+                        // towards the tail and the pick takes the freed place next to the active range.
+                        bool gate_hit = false, budget_hit = false, storage_hit = false;
+                        const int32_t* bk = p.bclass + grp.bclass_off;
+                        for (int kc = 0; kc < p.n_classes && !storage_hit; ++kc) {
+                            const int b_k = __ldg(bk + kc);
+                            for (int ak = 0; ak < b_k && qcnt[kc] > 0; ++ak) {
+                                if (nP == Acap) { storage_hit = true; break; }  // completed entries were squeezed out above
+                                const int q0 = head + nP;
+                                int pos = -1;
+                                uint64_t e = 0;
+                                for (int base = 0; base < nQ && pos < 0; base += 32) {
+                                    const int i = base + lane;
+                                    const uint64_t c = (i < nQ) ? RING(WR(q0 + i)) : 0;
+                                    const uint32_t m = __ballot_sync(FULL, i < nQ && entry_cls(c) == kc);
+                                    if (m) {
+                                        const int src = __ffs(m) - 1;
+                                        pos = base + src;
+                                        e = __shfl_sync(FULL, c, src);
+                                    }
+                                }
+                                if (pos < 0) break;  // cannot happen while the counts are right
+                                const int l = entry_l(e);
+                                if (!(kinf || a == 0 || l <= R)) { budget_hit = true; break; }
+                                if (G + l + 1 > M) { gate_hit = true; break; }
+                                for (int base = (pos - 1) & ~31; pos > 0 && base >= 0; base -= 32) {
+                                    const int i = base + lane;
+                                    const bool mv = i < pos;
+                                    uint64_t c = 0;
+                                    if (mv) c = RING(WR(q0 + i));
+                                    __syncwarp();
+                                    if (mv) RING(WR(q0 + i + 1)) = c;
+                                    __syncwarp();
+                                }
+                                const uint32_t sw = (uint32_t)(t + entry_o(e) - 1);
+                                if (lane == 0) {
+                                    RING(WR(q0)) = e;
+                                    STATE(WA(shead + nP)) = sw;
+                                    qcnt[kc] -= 1;
+                                }
+                                next_fin = min(next_fin, sw);
+                                if (lane == (nP >> bsh)) cmin = min(cmin, sw);
+                                Ndec++;
+                                nP++;
+                                nQ--;
+                                G += l + 1;
+                                if (!kinf) R -= min(l, R);
+                                a++;
+                                CADD(C_PREFILL_TOKENS, l);
+                                __syncwarp();
+                            }
+                        }
+                        if (gate_hit) CADD(C_GATE_BLOCKED, 1);
+                        if (budget_hit) CADD(C_BUDGET_BLOCKED, 1);
+                        if (storage_hit) { CADD(C_ACAP_BLOCKED, 1); status |= 1u; }
+                        q_l = -1;
+                        break;
+                    }
                     while (a < cap && nQ > 0) {
                         if (nP == Acap) {
                             if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room
@@ -551,6 +630,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                             Ndec--;
                         }
                         q_l = entry_l(e);
+                        if ((kClassFlow && policy == 4) && lane == 0) qcnt[entry_cls(e)] += 1;
                         nP--;
                         nQ++;
                         nev++;
@@ -558,6 +638,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                     if (pf_lo > nP) pf_lo = nP;
                     CADD(C_EVICTIONS, nev);
                     CADD(C_WASTED_TOKENS, wasted);
+                    __syncwarp();
                 }
 
                 // ---- process: one token per request whose prompt is in the cache; U_t = G

@@ -127,3 +127,7 @@ def test_config6_full_paper_setting():
     # never overflows, and nothing is dropped
     n = cfg.groups[0].n_replicas
     assert c[:n, I["overflow_steps"]].sum() == 0 and c[:, I["dropped"]].sum() == 0
+    # Algorithm 1 with b = (4,4,4) (last group): usage never passes sum_k b_k w_k = 16240 < M, no eviction (Thm. 3.3)
+    alg1 = c[3 * n:]
+    assert (alg1[:, I["max_U"]] <= 16240).all() and alg1[:, I["evictions"]].sum() == 0
+    assert alg1[:, I["gate_blocked_steps"]].sum() == 0 and alg1[:, I["completed"]].min() > 40000
