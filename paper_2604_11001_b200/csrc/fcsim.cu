@@ -164,30 +164,64 @@ __global__ void reduce_counters_kernel(const long long* __restrict__ counters, c
     }
 }
 
-// One block per chunk of replicas; thread b walks bins b, b+blockDim, .. (coalesced rows).
+// One block per chunk of replicas.  HBM-bound: every histogram word is read once (4 bytes per bin and
+// replica), 16 bytes per thread and load when the rows allow it (bins % 4 == 0), several loads in flight.
+template <int VEC>
 __global__ void reduce_hist_kernel(const int* __restrict__ hist, const DevGroup* __restrict__ groups, int n_groups,
                                    int n_replicas, int bins, int chunk, long long* __restrict__ out) {
     const int n_chunks = (n_replicas + chunk - 1) / chunk;
     for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
         const int r0 = c * chunk, r1 = min(n_replicas, r0 + chunk);
-        for (int b = threadIdx.x; b < bins; b += blockDim.x) {
+        for (int b = threadIdx.x * VEC; b < bins; b += blockDim.x * VEC) {
             int g = group_of(groups, n_groups, r0);
             int g_end = groups[g].first + groups[g].n;
-            long long acc = 0;
-            for (int r = r0; r < r1; ++r) {
+            long long acc[4] = {0, 0, 0, 0};
+            int r = r0;
+            while (r < r1) {
                 if (r >= g_end) {
-                    if (acc) atomicAdd(reinterpret_cast<unsigned long long*>(out + (size_t)g * bins + b),
-                                       (unsigned long long)acc);
-                    acc = 0;
+                    for (int v = 0; v < VEC; ++v) {
+                        if (acc[v]) atomicAdd(reinterpret_cast<unsigned long long*>(out + (size_t)g * bins + b + v),
+                                              (unsigned long long)acc[v]);
+                        acc[v] = 0;
+                    }
                     ++g;
                     g_end = groups[g].first + groups[g].n;
                 }
-                acc += hist[(size_t)r * bins + b];
+                const int stop = min(r1, g_end);
+                if (VEC == 4) {
+                    const int4* row = reinterpret_cast<const int4*>(hist + (size_t)r * bins + b);
+                    const size_t pitch = (size_t)bins / 4;
+                    int k = 0;
+                    for (; r + k + 4 <= stop; k += 4) {  // four independent 16-byte loads in flight
+                        const int4 x0 = __ldg(row + (size_t)(k + 0) * pitch), x1 = __ldg(row + (size_t)(k + 1) * pitch);
+                        const int4 x2 = __ldg(row + (size_t)(k + 2) * pitch), x3 = __ldg(row + (size_t)(k + 3) * pitch);
+                        acc[0] += (long long)x0.x + x1.x + x2.x + x3.x;
+                        acc[1] += (long long)x0.y + x1.y + x2.y + x3.y;
+                        acc[2] += (long long)x0.z + x1.z + x2.z + x3.z;
+                        acc[3] += (long long)x0.w + x1.w + x2.w + x3.w;
+                    }
+                    for (; r + k < stop; ++k) {
+                        const int4 x = __ldg(row + (size_t)k * pitch);
+                        acc[0] += x.x; acc[1] += x.y; acc[2] += x.z; acc[3] += x.w;
+                    }
+                } else {
+                    for (int q = r; q < stop; ++q) acc[0] += hist[(size_t)q * bins + b];
+                }
+                r = stop;
             }
-            if (acc) atomicAdd(reinterpret_cast<unsigned long long*>(out + (size_t)g * bins + b),
-                               (unsigned long long)acc);
+            for (int v = 0; v < VEC; ++v)
+                if (acc[v]) atomicAdd(reinterpret_cast<unsigned long long*>(out + (size_t)g * bins + b + v),
+                                      (unsigned long long)acc[v]);
         }
     }
+}
+
+void launch_reduce_hist(const int* hist, const DevGroup* groups, int G, int R, int bins, int blocks, long long* out,
+                        cudaStream_t st) {
+    if (bins % 4 == 0)
+        reduce_hist_kernel<4><<<blocks, std::min(256, bins / 4), 0, st>>>(hist, groups, G, R, bins, kStatsChunk, out);
+    else
+        reduce_hist_kernel<1><<<blocks, 256, 0, st>>>(hist, groups, G, R, bins, kStatsChunk, out);
 }
 
 }  // namespace
@@ -471,8 +505,7 @@ extern "C" int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_o
         }
         if (bins > 0) {
             const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
-            reduce_hist_kernel<<<blocks, 256, 0, st>>>(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins,
-                                                       kStatsChunk, d_hist);
+            launch_reduce_hist(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins, blocks, d_hist, st);
             CUDA_TRY(h, cudaGetLastError());
         }
         host_scratch.resize(bytes / 8);
@@ -543,8 +576,7 @@ extern "C" int fcsim_stats_noalloc(fcsim_t* h, void* cuda_stream, fcsim_summary*
     }
     if (bins > 0) {
         const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
-        reduce_hist_kernel<<<blocks, 256, 0, st>>>(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins,
-                                                   kStatsChunk, d_hist);
+        launch_reduce_hist(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins, blocks, d_hist, st);
         CUDA_TRY(h, cudaGetLastError());
     }
     CUDA_TRY(h, cudaMemcpyAsync(g_noalloc_host_rows, d_cnt, words * 8, cudaMemcpyDeviceToHost, st));

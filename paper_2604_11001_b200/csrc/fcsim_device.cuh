@@ -478,9 +478,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                     __syncwarp();
                 }
 
-                // ---- completed entries must be gone before an eviction (the newest entry has to be a live
-                //      one), before the active range runs out of storage, and when too many have piled up
-                bool squeeze = nD > 0 && (nD >= kCompactAt || G > M || ((kClassFlow && policy == 4) && nP + nQ > Acap));
+                // ---- completed entries are squeezed out when too many have piled up, before the active range
+                //      runs out of storage, and before the whole active range is sent back (alpha-protection)
+                bool squeeze = nD > 0 && (nD >= kCompactAt || (policy == 3 && G > M) ||
+                                          ((kClassFlow && policy == 4) && nP + nQ > Acap));
 
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
                 int a = 0;
@@ -616,10 +617,31 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                         cmin = kNoFin;
                         next_fin = kNoFin;
                     }
-                    while (policy != 3 && G > M && nP > 0) {
-                        const int i = nP - 1;
-                        const uint32_t sw = STATE(WA(shead + i));
-                        const uint64_t e = RING(WR(head + i));
+                    while (policy != 3 && G > M && nP > nD) {
+                        int i = nP - 1;
+                        uint32_t sw = STATE(WA(shead + i));
+                        if (sw == kDead) {
+                            // completed entries lie on top of the newest live one: find it (backwards, 32 at a
+                            // time), and move it to the top place, next to the queue, where it becomes the
+                            // queue head; its old place joins the completed entries
+                            int found = -1;
+                            for (int top = nP; found < 0 && top > 0; top -= 32) {
+                                const int idx = top - 32 + lane;
+                                const uint32_t w = (idx >= 0) ? STATE(WA(shead + idx)) : kDead;
+                                const uint32_t m = __ballot_sync(FULL, w != kDead);
+                                if (m) found = top - 1 - __clz(m);
+                            }
+                            i = found;
+                            sw = STATE(WA(shead + i));
+                            const uint64_t moved = RING(WR(head + i));
+                            __syncwarp();
+                            if (lane == 0) {
+                                RING(WR(head + nP - 1)) = moved;
+                                STATE(WA(shead + i)) = kDead;
+                            }
+                            __syncwarp();
+                        }
+                        const uint64_t e = RING(WR(head + nP - 1));
                         if (sw & kPrefillBit) {
                             G -= (int)(sw & ~kPrefillBit);
                             n_pref--;
