@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -24,6 +25,7 @@ constexpr int kStatsChunk = 256;             // replicas reduced by one block be
 struct Layout {
     int RC, Apad, S;
     size_t ws_stride, smem_per_warp, qcnt_off;  // qcnt_off: per-class queue counts (Algorithm 1), 0 = unused
+    size_t tstage_off;                          // trace staging buffers, 0 = unused
     int warps_per_block;
     int n_rec;
     long long R;
@@ -94,6 +96,15 @@ int plan(const fcsim_config* c, Layout* L) {
     L->qcnt_off = (size_t)L->RC * 8 + (size_t)L->Apad * 4 + (size_t)L->S * 8;
     L->smem_per_warp = L->qcnt_off + (any_classflow ? align_up((size_t)c->n_classes * 4, 16) : 0);
     if (!any_classflow) L->qcnt_off = 0;
+    // Optional trace staging (environment FCSIM_TRACE_BULK=1): 2 x 32 records of 8 bytes in shared memory,
+    // each full block leaving with one 256-byte bulk copy.  Off by default: measured slower than keeping
+    // the records in registers (the stream is 8 bytes per slot, and the extra shared memory costs a CTA).
+    L->tstage_off = 0;
+    const char* tb = getenv("FCSIM_TRACE_BULK");
+    if (c->trace_stride > 0 && tb && tb[0] == '1') {
+        L->tstage_off = L->smem_per_warp;
+        L->smem_per_warp += 512;
+    }
     if (L->smem_per_warp > kSmemBudget) return FCSIM_ECAP;
     int w = kWarpsPerBlock;
     while (w > 1 && (size_t)w * L->smem_per_warp > kSmemBudget) w >>= 1;
@@ -429,6 +440,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.gpool = h->d_gpool;
     p.bclass = h->d_bclass;
     p.qcnt_off = (uint32_t)L.qcnt_off;
+    p.tstage_off = (uint32_t)L.tstage_off;
     p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
     p.workspace = static_cast<unsigned char*>(b->workspace);
     p.ws_stride = L.ws_stride;

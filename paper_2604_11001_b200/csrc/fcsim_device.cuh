@@ -73,6 +73,8 @@ struct Params {
     const unsigned short* gpool;  // guide tables: for bucket b of the top bits of u, the first candidate index
     const int32_t* bclass;        // per-class budgets b_k of the Algorithm-1 groups
     uint32_t qcnt_off;            // byte offset of the per-class queue counts in a warp's shared memory (0 = none)
+    uint32_t tstage_off;          // byte offset of the trace staging area (2 x 32 records) in a warp's shared
+                                  // memory; 0 = records are kept in registers and stored with plain stores
     const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
     const DevArrivals* arrivals;
     const DevGroup* groups;
@@ -124,6 +126,21 @@ __device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, c
     }
     return tb.vmin + (int)lo;
 }
+
+// Bulk asynchronous copy shared -> global of one staged block of trace records (TMA engine, no tensor map).
+// Both addresses must be 16-byte aligned and the size a multiple of 16; the caller checks that.
+__device__ __forceinline__ void bulk_store_commit(void* gdst, const void* ssrc, uint32_t bytes) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(ssrc);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // staged records visible to the async proxy
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(s), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Wait until at most `pending` of this thread's bulk copies have not finished READING their source.
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t lanemask_lt() {
     uint32_t m;
@@ -299,6 +316,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
         int cd = stride > 0 ? stride - (t % stride) : 0;
         const int rec_lo = rec;
         int tr_u = 0, tr_q = 0;
+        // staged variant: records go to shared memory (two buffers of 32) and every full block of 32 leaves
+        // with one 256-byte bulk copy issued by lane 0, when the row's address allows it
+        int2* tstage = reinterpret_cast<int2*>(my + p.tstage_off);
+        const bool staged = p.tstage_off != 0 && stride > 0 &&
+                            ((reinterpret_cast<uintptr_t>(p.trace + (size_t)r * p.n_rec) & 15u) == 0);
         int2* trow = p.trace ? p.trace + (size_t)r * p.n_rec : nullptr;
         int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
         int2* lrow = p.complog ? p.complog + (size_t)r * p.complog_cap : nullptr;
@@ -726,10 +748,27 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
                 maxQ = max(maxQ, nQ);
                 if (stride > 0 && --cd == 0) {
                     cd = stride;
-                    if (lane == (rec & 31)) { tr_u = G; tr_q = nQ; }
-                    if ((rec & 31) == 31) {
-                        const int b0 = rec & ~31;
-                        if (b0 + lane >= rec_lo) TROW(b0 + lane) = make_int2(tr_u, tr_q);
+                    if (staged) {
+                        if (lane == 0) tstage[rec & 63] = make_int2(G, nQ);
+                        if ((rec & 31) == 31) {
+                            const int b0 = rec & ~31;
+                            __syncwarp();
+                            if (b0 >= rec_lo) {
+                                if (lane == 0) {
+                                    bulk_store_commit(trow + b0, tstage + (b0 & 32), 256u);
+                                    bulk_wait_read<1>();  // the other buffer (copy issued 32 records ago) is free again
+                                }
+                            } else if (b0 + lane >= rec_lo) {
+                                TROW(b0 + lane) = tstage[(b0 & 32) + lane];  // block begun by an earlier launch
+                            }
+                            __syncwarp();
+                        }
+                    } else {
+                        if (lane == (rec & 31)) { tr_u = G; tr_q = nQ; }
+                        if ((rec & 31) == 31) {
+                            const int b0 = rec & ~31;
+                            if (b0 + lane >= rec_lo) TROW(b0 + lane) = make_int2(tr_u, tr_q);
+                        }
                     }
                     rec++;
                 }
@@ -740,7 +779,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_ste
         // ------------------------------------------------------------------ flush, final extras, spill
         if (stride > 0 && (rec & 31) != 0) {
             const int b0 = rec & ~31;
-            if (b0 + lane >= rec_lo && b0 + lane < rec) TROW(b0 + lane) = make_int2(tr_u, tr_q);
+            if (staged) {
+                __syncwarp();
+                if (b0 + lane >= rec_lo && b0 + lane < rec) TROW(b0 + lane) = tstage[(b0 & 32) + lane];
+            } else if (b0 + lane >= rec_lo && b0 + lane < rec) {
+                TROW(b0 + lane) = make_int2(tr_u, tr_q);
+            }
+        }
+        if (staged) {  // the staging buffers are reused by the next replica and the copies must land before the exit
+            if (lane == 0) bulk_wait_all();
+            __syncwarp();
         }
         long long age = 0, resj = 0;
         for (int i = lane; i < nP + nQ; i += 32) {

@@ -138,3 +138,13 @@ def test_large_active_set_and_lazy_removal_paths():
     assert_same(tight, run_gpu(tight), ref, 1500, "storage-bound")
     churn = wl.config2(replicas=2, T=3000).with_(M=20000, Acap=96)
     assert_same(churn, run_gpu(churn, pieces=[1000, 1, 1999]), orc.run(churn), 3000, "eviction churn")
+
+
+def test_trace_bulk_copy_variant(monkeypatch):
+    # opt-in variant: trace records staged in shared memory and stored with 256-byte bulk copies.  Rows of 333
+    # records: odd rows start 8 bytes off a 16-byte boundary and must fall back to plain stores.
+    monkeypatch.setenv("FCSIM_TRACE_BULK", "1")
+    cfg = wl.config1(replicas=9, T=333)
+    assert_same(cfg, run_gpu(cfg, pieces=[100, 7, 226]), orc.run(cfg), 333, "bulk trace")
+    cfg = wl.config2(replicas=2, T=2000)
+    assert_same(cfg, run_gpu(cfg), orc.run(cfg), 2000, "bulk trace cfg2")
