@@ -148,3 +148,36 @@ def test_trace_bulk_copy_variant(monkeypatch):
     assert_same(cfg, run_gpu(cfg, pieces=[100, 7, 226]), orc.run(cfg), 333, "bulk trace")
     cfg = wl.config2(replicas=2, T=2000)
     assert_same(cfg, run_gpu(cfg), orc.run(cfg), 2000, "bulk trace cfg2")
+
+
+def test_maximum_sizes():
+    # lengths at the 16-bit limit, capacity 2^30, rings so large that a CTA holds a single warp,
+    # 255 arrivals in a slot, the largest flow rate
+    big = wl.SimConfig(
+        M=1 << 30, K=0, T_max=300, Qcap=9000, Acap=8000, seed=(1 << 63) + 5, class_law=wl.constant_table(0),
+        prompt=(wl.uniform_table(65000, 65535),), decode=(wl.table_from_pmf(1, [0.5] + [0.0] * 65533 + [0.5]),),
+        arrivals=(wl.Arrivals((wl.table_from_pmf(0, [0.5] + [0.0] * 254 + [0.5]),)),),
+        groups=(wl.Group(wl.POLICY_FLOW, b_fp=0xFFFFFFFF, n_replicas=3),
+                wl.Group(wl.POLICY_GREEDY, n_replicas=3, rng_replica_base=0xFFFFFFF0)),
+        trace_stride=1, hist_bins=4, hist_shift=30, complog_cap=100000)
+    gpu = run_gpu(big)
+    assert gpu["launch"]["warps_per_block"] == 1
+    ref = orc.run(big)
+    assert_same(big, gpu, ref, 300, "maximum sizes")
+    assert ref["counters"][:, orc.CIDX["max_U"]].max() > 1 << 28
+    assert ref["counters"][:, orc.CIDX["dropped"]].sum() > 0
+
+
+def test_horizon_limit_and_range_errors():
+    from paper_2604_11001_b200 import binding as fb
+    cfg = wl.config1(replicas=2, T=50)
+    sim = fb.Simulation(cfg)
+    sim.run(50)
+    with pytest.raises(fb.FcsimError) as e:
+        sim.run(1)
+    assert e.value.code == -4
+    assert sim.steps_done == 50
+    sim.close()
+    # slots close to the 24-bit horizon limit: arrival times near 2^24 must survive the packing
+    late = wl.config1(replicas=2, T=(1 << 24) - 1)
+    assert fb.fcsim_query_sizes(late.with_(trace_stride=0, complog_cap=0))["trace"] == 0
