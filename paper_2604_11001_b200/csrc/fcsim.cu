@@ -405,7 +405,13 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
 
     const size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
     if (smem_block > (size_t)prop.sharedMemPerBlockOptin) return fail(FCSIM_ECAP);
-    h->kernel = L.qcnt_off ? fcsim_step_kernel<true> : fcsim_step_kernel<false>;
+    // six CTAs per SM need <= 80 registers per thread and their shared memory (plus 1 KB each that the
+    // system reserves) within the SM's 228 KB; otherwise the 5-CTA register allocation is the better one
+    const bool six = 6 * (smem_block + 1024) <= (size_t)prop.sharedMemPerMultiprocessor;
+    if (L.qcnt_off)
+        h->kernel = six ? fcsim_step_kernel<true, 6> : fcsim_step_kernel<true, 5>;
+    else
+        h->kernel = six ? fcsim_step_kernel<false, 6> : fcsim_step_kernel<false, 5>;
     e = cudaFuncSetAttribute(h->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block);
     if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
     int occ = 0;

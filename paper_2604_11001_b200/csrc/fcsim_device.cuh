@@ -207,15 +207,12 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define HROW(i) hrow[(i)]
 #endif
 
-// Minimum resident CTAs per SM the compiler must allow for (bounds registers per thread).
-#ifndef FCSIM_MIN_CTAS
-#define FCSIM_MIN_CTAS 5
-#endif
-
 // kClassFlow: compiled with the per-class activation of Algorithm 1 (policy 4); the variant without it is
 // used when no group asks for it, so that the common policies do not carry its code.
-template <bool kClassFlow>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32, FCSIM_MIN_CTAS) fcsim_step_kernel(const Params p) {
+// kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80 with a
+// few spilled words).  The host picks 6 when the shared memory of six CTAs fits the SM, else 5.
+template <bool kClassFlow, int kMinCtas>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
