@@ -43,7 +43,8 @@ struct orc_arrivals {
 };
 struct orc_group {
     int32_t policy;  // 0 FLOW, 1 GREEDY, 2 CHUNKED, 3 ALPHA (alpha-protection greedy, Section 4.1),
-                     // 4 CLASSFLOW (Algorithm 1: per-class budgets b_k, FIFO within a class)
+                     // 4 CLASSFLOW (Algorithm 1: per-class budgets b_k, FIFO within a class),
+                     // 5 MC (memory-constrained first-come-first-served benchmark of Section 4.1)
     uint32_t b_fp;
     int32_t chunk;
     int32_t arrivals_id;
@@ -51,6 +52,8 @@ struct orc_group {
     int32_t n_replicas;
     int32_t m_admit;  // ALPHA: a new prompt is admitted only while usage stays <= m_admit = (1-alpha) M
     const int32_t* b_class;  // CLASSFLOW (policy 4, Algorithm 1): activation budget b_k of every class
+    int32_t mc_worst_case;   // MC: 0 = output lengths known, 1 = every request is projected with the longest
+                             //     output length of its class (the unknown-length adaptation of Section 4.1)
 };
 struct orc_config {
     int32_t M, K, T_max, Qcap, Acap;
@@ -126,9 +129,33 @@ constexpr uint32_t STREAM_ARR = 1;
 struct Request {
     int64_t id;
     int32_t cls, l, o, t_arr;
+    int32_t o_proj;  // output length assumed when future memory is projected (MC benchmark)
     int32_t p;  // prompt tokens in the cache
     int32_t j;  // output tokens generated
 };
+
+// MC benchmark (Section 4.1): "only activates requests if the future memory usage remains within the
+// memory limit".  With no further activation, an active request that has generated j tokens before slot t
+// holds l + j + (tau - t + 1) tokens in slot tau until the slot of its (projected) last token,
+// tau_end = t + (o_proj - j) - 1, and nothing afterwards.  The candidate h would start in slot t.
+// The usage only drops when a request ends, so it is enough to look at every request's last slot.
+bool fits_future(const std::vector<Request>& P, const Request& h, int32_t t, int64_t M) {
+    std::vector<Request> all(P);
+    Request c = h;
+    c.p = c.l;
+    c.j = 0;
+    all.push_back(c);
+    for (const Request& e : all) {
+        const int64_t tau = (int64_t)t + (e.o_proj - e.j) - 1;  // last slot of e
+        int64_t usage = 0;
+        for (const Request& r : all) {
+            const int64_t r_end = (int64_t)t + (r.o_proj - r.j) - 1;
+            if (r_end >= tau) usage += (int64_t)r.l + r.j + (tau - t + 1);
+        }
+        if (usage > M) return false;
+    }
+    return true;
+}
 
 int64_t kv_usage(const std::vector<Request>& P) {
     int64_t u = 0;
@@ -161,7 +188,8 @@ int validate(const orc_config& c) {
     }
     for (int g = 0; g < c.n_groups; ++g) {
         const orc_group& G = c.groups[g];
-        if (G.policy < 0 || G.policy > 4 || G.n_replicas < 1) return -1;
+        if (G.policy < 0 || G.policy > 5 || G.n_replicas < 1) return -1;
+        if (G.policy == 5 && (G.mc_worst_case < 0 || G.mc_worst_case > 1)) return -1;
         if (G.policy == 4) {
             if (!G.b_class) return -1;
             for (int k = 0; k < c.n_classes; ++k)
@@ -184,7 +212,7 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
     const orc_arrivals& arr = cfg.arrivals[grp.arrivals_id];
     const int64_t INF = std::numeric_limits<int64_t>::max() / 4;
     const bool flow = grp.policy == 0, chunked = grp.policy == 2, alpha = grp.policy == 3;
-    const bool classflow = grp.policy == 4;
+    const bool classflow = grp.policy == 4, mc = grp.policy == 5;
     const int64_t M = cfg.M;
     // alpha-protection greedy (Section 4.1): a new prompt with initial memory l+1 joins only if the usage
     // stays within (1-alpha) M; every other policy admits up to the capacity itself
@@ -219,6 +247,8 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
             r.t_arr = t;
             r.p = 0;
             r.j = 0;
+            r.o_proj = r.o;
+            if (mc && grp.mc_worst_case) r.o_proj = cfg.decode[r.cls].vmin + (int32_t)cfg.decode[r.cls].n - 1;
             if (arrcls) arrcls[(int64_t)(t - 1) * cfg.n_classes + r.cls]++;
             C[C_ARRIVED]++;
             if ((int64_t)Q.size() >= (int64_t)cfg.Qcap) {
@@ -303,6 +333,7 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
                 need = (int64_t)h.l + 1;
             }
             if (G + need > admit_limit) { C[C_GATE_BLOCKED]++; break; }
+            if (mc && !fits_future(P, h, t, M)) { C[C_GATE_BLOCKED]++; break; }
             Q.pop_front();
             h.p = (int32_t)g;
             h.j = 0;

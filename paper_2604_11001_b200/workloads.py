@@ -31,6 +31,7 @@ POLICY_GREEDY = 1
 POLICY_CHUNKED = 2
 POLICY_ALPHA = 3   # alpha-protection greedy (Section 4.1)
 POLICY_CLASSFLOW = 4   # Algorithm 1: per-class activation budgets b_k, FIFO within a class
+POLICY_MC = 5          # memory-constrained FCFS benchmark (Section 4.1): admit only if future usage stays <= M
 
 _TWO32 = float(2 ** 32)
 
@@ -165,6 +166,7 @@ class Group:
     n_replicas: int = 1
     m_admit: int = 0           # ALPHA: admission keeps usage <= m_admit = floor((1 - alpha) M)
     b_class: Tuple[int, ...] = ()  # CLASSFLOW: integer budget b_k of every class (Algorithm 1)
+    mc_worst_case: int = 0         # MC: 1 = project every request with its class's longest output length
 
 
 @dataclass(frozen=True)
@@ -369,11 +371,12 @@ def random_small_config(seed: int, n_replicas: int = 4, T: int = 60) -> SimConfi
                                      (int(rng.integers(0, 2 ** 31)), int(rng.integers(0, 2 ** 31)))))
     groups = []
     base = 0
-    for pol in (POLICY_FLOW, POLICY_GREEDY, POLICY_CHUNKED, POLICY_ALPHA, POLICY_CLASSFLOW):
+    for pol in (POLICY_FLOW, POLICY_GREEDY, POLICY_CHUNKED, POLICY_ALPHA, POLICY_CLASSFLOW, POLICY_MC):
         groups.append(Group(pol, b_fp=int(rng.integers(0, 3 * 65536)), chunk=int(rng.integers(1, 9)),
                             arrivals_id=int(rng.integers(0, 2)), rng_replica_base=base,
                             n_replicas=n_replicas, m_admit=int(rng.integers(max(2, M // 2), M + 1)),
-                            b_class=tuple(int(x) for x in rng.integers(0, 3, size=n_classes))))
+                            b_class=tuple(int(x) for x in rng.integers(0, 3, size=n_classes)),
+                            mc_worst_case=int(rng.integers(0, 2))))
         base += int(rng.integers(0, 2)) * n_replicas
     stride = int(rng.choice([1, 1, 2, 3]))
     return SimConfig(

@@ -8,7 +8,7 @@ import numpy as np
 from paper_2604_11001_b200 import workloads as wl
 
 POLICIES = {"flow": wl.POLICY_FLOW, "greedy": wl.POLICY_GREEDY, "chunked": wl.POLICY_CHUNKED,
-            "alpha": wl.POLICY_ALPHA}
+            "alpha": wl.POLICY_ALPHA, "mc": wl.POLICY_MC}
 
 
 def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, ma=0, **extra):

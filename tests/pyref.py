@@ -77,7 +77,11 @@ def brute_force(cfg, replica, n_steps):
             if len(waiting()) >= cfg.Qcap:
                 cnt["dropped"] += 1
             else:
-                reqs.append(dict(id=len(reqs), cls=cls, l=l, o=o, t_arr=t, status="wait", act_seq=None, p=0, j=0))
+                o_proj = o
+                if grp.policy == 5 and grp.mc_worst_case:
+                    o_proj = cfg.decode[cls].vmin + len(cfg.decode[cls].cdf) - 1
+                reqs.append(dict(id=len(reqs), cls=cls, l=l, o=o, o_proj=o_proj, t_arr=t, status="wait",
+                                 act_seq=None, p=0, j=0))
         n_dec_start = sum(1 for r in active() if r["p"] == r["l"])
         room = None if cfg.K == 0 else (max(0, cfg.K - n_dec_start) if grp.policy == 2 else cfg.K)
         if grp.policy == 2:
@@ -142,6 +146,21 @@ def brute_force(cfg, replica, n_steps):
                     cnt["budget_blocked_steps"] += 1
                     break
                 need = g + 1
+            if grp.policy == 5:
+                # MC benchmark: run the system forward with no further arrivals or activations and look at
+                # the usage of every slot until everything has (by projection) finished
+                proj = [dict(l=r["l"], j=r["j"], left=r["o_proj"] - r["j"]) for r in active()]
+                proj.append(dict(l=h["l"], j=0, left=h["o_proj"]))
+                ok = True
+                while proj and ok:
+                    for q in proj:
+                        q["j"] += 1
+                        q["left"] -= 1
+                    ok = sum(q["l"] + q["j"] for q in proj) <= cfg.M
+                    proj = [q for q in proj if q["left"] > 0]
+                if not ok:
+                    cnt["gate_blocked_steps"] += 1
+                    break
             limit = grp.m_admit if grp.policy == 3 else cfg.M   # alpha-protection: keep usage <= (1-alpha) M
             if prospective() + need > limit:
                 cnt["gate_blocked_steps"] += 1

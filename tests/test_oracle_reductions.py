@@ -107,3 +107,33 @@ def test_alpha_protection_evicts_everything_on_overflow():
     # admission never takes the usage of an admission slot past the protection limit + growth of that slot:
     # max_U can exceed m_admit only through decoding growth, never beyond M
     assert (c[:, I["max_U"]] <= cfg.M).all()
+
+
+def test_mc_benchmark_never_overflows_and_equals_greedy_when_memory_is_ample():
+    # Section 4.1's MC benchmark admits only what provably fits until completion: no slot can overflow, so
+    # nothing is ever evicted, whatever the load
+    for cfg in (wl.config1(replicas=3, T=2500), wl.config5(replicas=2, T=4000).with_(trace_stride=1)):
+        n = cfg.groups[0].n_replicas
+        for worst in (0, 1):
+            mc = cfg.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=n, mc_worst_case=worst),))
+            c = orc.run(mc, complog=False)["counters"]
+            assert c[:, I["evictions"]].sum() == 0 and c[:, I["overflow_steps"]].sum() == 0
+            assert (c[:, I["max_U"]] <= cfg.M).all() and c[:, I["completed"]].min() > 0
+    # with ample memory the projection never refuses and the policy is plain greedy
+    roomy = wl.config1(replicas=3, T=1500).with_(M=1 << 24)
+    mc = roomy.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=3),))
+    gr = roomy.with_(groups=(wl.Group(wl.POLICY_GREEDY, n_replicas=3),))
+    _same(orc.run(mc), orc.run(gr))
+
+
+def test_mc_worst_case_projection_equals_known_lengths_when_lengths_are_constant():
+    # the unknown-length adaptation projects with the longest output of the class; with one possible length it
+    # is the known-length rule, and with variable lengths it is more conservative (never more admissions)
+    cfg = wl.config6(replicas=2, T=2500).with_(M=2000)
+    known = cfg.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=2, mc_worst_case=0),))
+    worst = cfg.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=2, mc_worst_case=1),))
+    _same(orc.run(known), orc.run(worst))
+    var = wl.config1(replicas=3, T=2500)
+    k = orc.run(var.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=3, mc_worst_case=0),)), complog=False)
+    w = orc.run(var.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=3, mc_worst_case=1),)), complog=False)
+    assert (w["counters"][:, I["sum_U"]] < k["counters"][:, I["sum_U"]]).all()
