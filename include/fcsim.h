@@ -48,9 +48,13 @@ enum {
  * requests of that class are activated, first come first served within the class.  The memory gate, the
  * token budget and the last-in-first-out eviction are those of Algorithm 2 (they never act when the
  * condition of Theorem 3.3 holds); a pick that does not fit ends the loop of its class only. */
+/* MC is the memory-constrained benchmark of Section 4.1: first come first served, a request starts only if,
+ * with every running request and the candidate run to completion and nothing else started, the usage of every
+ * future slot stays within M (so no slot can overflow and nothing is evicted).  With mc_worst_case = 1 every
+ * request is projected with the longest output length of its class (the unknown-length adaptation). */
 enum {
     FCSIM_POLICY_FLOW = 0, FCSIM_POLICY_GREEDY = 1, FCSIM_POLICY_CHUNKED = 2, FCSIM_POLICY_ALPHA = 3,
-    FCSIM_POLICY_CLASSFLOW = 4
+    FCSIM_POLICY_CLASSFLOW = 4, FCSIM_POLICY_MC = 5
 };
 
 /* Integer inverse-CDF table.  Support {vmin .. vmin+n-1}; cdf[k] = floor(P(X <= vmin+k) * 2^32) clamped
@@ -81,7 +85,8 @@ typedef struct {
  *       common random numbers).
  * m_admit: ALPHA only, the admission limit floor((1 - alpha) M) in tokens, 1 .. M.
  * b_class: CLASSFLOW only, HOST array [n_classes] of the integer budgets b_k (0 .. 65535), borrowed during
- *       fcsim_create / fcsim_query_sizes; NULL otherwise. */
+ *       fcsim_create / fcsim_query_sizes; NULL otherwise.
+ * mc_worst_case: MC only, 0 = output lengths known, 1 = project with the class's longest output length. */
 typedef struct {
     int32_t policy;
     uint32_t b_fp;
@@ -91,6 +96,7 @@ typedef struct {
     int32_t n_replicas;
     int32_t m_admit;
     const int32_t* b_class;
+    int32_t mc_worst_case;
 } fcsim_group;
 
 /* M: KV capacity in tokens (1 .. 2^30).  K: prefill-token budget per slot, 0 = none (the paper's model).

@@ -26,6 +26,8 @@ struct Layout {
     int RC, Apad, S;
     size_t ws_stride, smem_per_warp, qcnt_off;  // qcnt_off: per-class queue counts (Algorithm 1), 0 = unused
     size_t tstage_off;                          // trace staging buffers, 0 = unused
+    size_t state_bytes;                         // ring + state words (+ projection words) saved between launches
+    int has_v;
     int warps_per_block;
     int n_rec;
     long long R;
@@ -68,10 +70,14 @@ int plan(const fcsim_config* c, Layout* L) {
         }
     }
     long long R = 0;
-    bool any_classflow = false;
+    bool any_classflow = false, any_mc = false;
     for (int g = 0; g < c->n_groups; ++g) {
         const fcsim_group& G = c->groups[g];
-        if (G.policy < 0 || G.policy > 4 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.policy < 0 || G.policy > 5 || G.n_replicas < 1) return FCSIM_EINVAL;
+        if (G.policy == FCSIM_POLICY_MC) {
+            if (G.mc_worst_case < 0 || G.mc_worst_case > 1) return FCSIM_EINVAL;
+            any_mc = true;
+        }
         if (G.policy == FCSIM_POLICY_CLASSFLOW) {
             if (!G.b_class) return FCSIM_EINVAL;
             for (int k = 0; k < c->n_classes; ++k)
@@ -92,8 +98,11 @@ int plan(const fcsim_config* c, Layout* L) {
     L->RC = (int)align_up((size_t)rc, 2);
     L->Apad = (int)align_up((size_t)c->Acap, 4);
     L->S = (int)align_up((size_t)std::max(128, max_count), 2);
-    L->ws_stride = kHeaderWords * 4 + (size_t)L->RC * 8 + (size_t)L->Apad * 4;
-    L->qcnt_off = (size_t)L->RC * 8 + (size_t)L->Apad * 4 + (size_t)L->S * 8;
+    // the MC benchmark keeps one more word per active entry (projected usage in its last slot), saved with the state
+    L->state_bytes = (size_t)L->RC * 8 + (size_t)L->Apad * 4 * (any_mc ? 2 : 1);
+    L->has_v = any_mc ? 1 : 0;
+    L->ws_stride = kHeaderWords * 4 + L->state_bytes;
+    L->qcnt_off = L->state_bytes + (size_t)L->S * 8;
     L->smem_per_warp = L->qcnt_off + (any_classflow ? align_up((size_t)c->n_classes * 4, 16) : 0);
     if (!any_classflow) L->qcnt_off = 0;
     // Optional trace staging (environment FCSIM_TRACE_BULK=1): 2 x 32 records of 8 bytes in shared memory,
@@ -326,7 +335,8 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
             bclass.insert(bclass.end(), G.b_class, G.b_class + c->n_classes);
         }
         grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas,
-                           G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M, boff, 0};
+                           G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M, boff,
+                           G.policy == FCSIM_POLICY_MC ? G.mc_worst_case : 0};
         first += G.n_replicas;
     }
     CUDA_TRY(h, cudaMalloc(&h->d_bclass, bclass.size() * sizeof(int32_t)));
@@ -408,7 +418,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     // six CTAs per SM need <= 80 registers per thread and their shared memory (plus 1 KB each that the
     // system reserves) within the SM's 228 KB; otherwise the 5-CTA register allocation is the better one
     const bool six = 6 * (smem_block + 1024) <= (size_t)prop.sharedMemPerMultiprocessor;
-    if (L.qcnt_off)
+    if (L.qcnt_off || L.has_v)
         h->kernel = six ? fcsim_step_kernel<true, 6> : fcsim_step_kernel<true, 5>;
     else
         h->kernel = six ? fcsim_step_kernel<false, 6> : fcsim_step_kernel<false, 5>;
@@ -447,6 +457,8 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.bclass = h->d_bclass;
     p.qcnt_off = (uint32_t)L.qcnt_off;
     p.tstage_off = (uint32_t)L.tstage_off;
+    p.state_bytes = (uint32_t)L.state_bytes;
+    p.has_v = L.has_v;
     p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
     p.workspace = static_cast<unsigned char*>(b->workspace);
     p.ws_stride = L.ws_stride;

@@ -60,7 +60,7 @@ struct DevGroup {
     int32_t n;
     int32_t admit_limit;  // usage a new admission may reach: M, or (1-alpha) M for the alpha-protection policy
     int32_t bclass_off;   // Algorithm 1: index of the group's per-class budgets in Params::bclass
-    int32_t pad;
+    int32_t mc_worst;     // MC benchmark: project with the class's longest output length
 };
 
 struct Params {
@@ -73,6 +73,8 @@ struct Params {
     const unsigned short* gpool;  // guide tables: for bucket b of the top bits of u, the first candidate index
     const int32_t* bclass;        // per-class budgets b_k of the Algorithm-1 groups
     uint32_t qcnt_off;            // byte offset of the per-class queue counts in a warp's shared memory (0 = none)
+    uint32_t state_bytes;         // ring + state words (+ projection words): what is saved between launches
+    int32_t has_v;                // 1 = a projection word per active entry follows the state words (MC benchmark)
     uint32_t tstage_off;          // byte offset of the trace staging area (2 x 32 records) in a warp's shared
                                   // memory; 0 = records are kept in registers and stored with plain stores
     const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
@@ -207,11 +209,12 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define HROW(i) hrow[(i)]
 #endif
 
-// kClassFlow: compiled with the per-class activation of Algorithm 1 (policy 4); the variant without it is
-// used when no group asks for it, so that the common policies do not carry its code.
+// kExt: compiled with the per-class activation of Algorithm 1 (policy 4) and the future-memory test of the
+// MC benchmark (policy 5); the variant without them is used when no group asks for either, so that the
+// common policies do not carry their code.
 // kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80 with a
 // few spilled words).  The host picks 6 when the shared memory of six CTAs fits the SM, else 5.
-template <bool kClassFlow, int kMinCtas>
+template <bool kExt, int kMinCtas>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
@@ -219,8 +222,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
     unsigned char* my = smem_raw + (size_t)warp * p.smem_per_warp;
     uint64_t* ring = reinterpret_cast<uint64_t*>(my);
     uint32_t* state = reinterpret_cast<uint32_t*>(my + (size_t)p.RC * 8);
-    uint64_t* stage = reinterpret_cast<uint64_t*>(my + (size_t)p.RC * 8 + (size_t)p.Apad * 4);
-    const int state_bytes = p.RC * 8 + p.Apad * 4;  // multiple of 16 (host guarantees)
+    // MC benchmark: vproj[k] = memory usage projected for the last slot of active entry k (same ring as state)
+    int* vproj = reinterpret_cast<int*>(state + p.Apad);
+    const int state_bytes = (int)p.state_bytes;  // multiple of 16 (host guarantees)
+    uint64_t* stage = reinterpret_cast<uint64_t*>(my + state_bytes);
     uint32_t* qcnt = reinterpret_cast<uint32_t*>(my + p.qcnt_off);  // waiting requests per class (Algorithm 1 only)
 
     const int RC = p.RC, Acap = p.Acap, Qcap = p.Qcap, M = p.M, K = p.K, S = p.S;
@@ -336,11 +341,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 const uint32_t m = __ballot_sync(FULL, dead);
                 const int sh = holes + __popc(m & gt_mask);  // completed entries after this one
                 const bool mv = valid && !dead && sh > 0;
+                int v = 0;
                 if (mv) e = RING(WR(head + i));
+                if (kExt && p.has_v && mv) v = vproj[WA(shead + i)];
                 __syncwarp();
                 if (mv) {
                     RING(WR(head + i + sh)) = e;
                     STATE(WA(shead + i + sh)) = sw;
+                    if (kExt && p.has_v) vproj[WA(shead + i + sh)] = v;
                 }
                 __syncwarp();
                 holes += __popc(m);
@@ -363,7 +371,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             next_fin = __reduce_min_sync(FULL, cmin);
         };
         rebuild_minima();
-        if ((kClassFlow && policy == 4)) {  // Algorithm 1 picks per class: count the waiting requests of every class
+        if ((kExt && policy == 4)) {  // Algorithm 1 picks per class: count the waiting requests of every class
             for (int c = lane; c < p.n_classes; c += 32) qcnt[c] = 0;
             __syncwarp();
             for (int i = lane; i < nQ; i += 32) atomicAdd(&qcnt[entry_cls(RING(WR(head + nP + i)))], 1u);
@@ -441,7 +449,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         for (int i = lane; i < acc; i += 32) {
                             const uint64_t e = STAGE(sp + i);
                             RING(WR(tail + i)) = e;
-                            if ((kClassFlow && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
+                            if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
                         }
                         nQ += acc;
                         __syncwarp();
@@ -500,14 +508,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 // ---- completed entries are squeezed out when too many have piled up, before the active range
                 //      runs out of storage, and before the whole active range is sent back (alpha-protection)
                 bool squeeze = nD > 0 && (nD >= kCompactAt || (policy == 3 && G > M) ||
-                                          ((kClassFlow && policy == 4) && nP + nQ > Acap));
+                                          ((kExt && policy == 4) && nP + nQ > Acap));
 
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
                 int a = 0;
                 const int cap = (policy == 0) ? B_t : 0x7fffffff;
                 for (;;) {
                     if (squeeze) { compact(); rebuild_minima(); squeeze = false; }
-                    if ((kClassFlow && policy == 4)) {
+                    if ((kExt && policy == 4)) {
                         // Algorithm 1: for every class k, up to b_k waiting requests of that class, oldest first.
                         // The pick leaves the middle of the queue: the entries ahead of it move one place
                         // towards the tail and the pick takes the freed place next to the active range.
@@ -585,6 +593,51 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             need = l + 1;
                         }
                         if (G + need > admit_limit) { CADD(C_GATE_BLOCKED, 1); break; }
+                        if (kExt && policy == 5) {
+                            // MC benchmark (Section 4.1): start the queue head only if the usage of every future
+                            // slot stays within M.  With a_i = l_i - (activation slot) + 1, request i holds a_i + tau
+                            // in slot tau up to its last slot f_i; the usage can only peak in some last slot.
+                            // vproj[k] holds the usage of slot f_k for the running requests, so the head h
+                            // (last slot f_h) fits iff vproj[k] + a_h + f_k <= M for every k with f_k <= f_h and
+                            // the usage of slot f_h itself, sum over f_i >= f_h of (a_i + f_h) + a_h + f_h, is <= M.
+                            const uint64_t eh = RING(WR(head + nP));
+                            const bool worst = grp.mc_worst != 0;
+                            const int op_h = worst ? (p.tables[1 + p.n_classes + entry_cls(eh)].vmin +
+                                                      (int)p.tables[1 + p.n_classes + entry_cls(eh)].n - 1)
+                                                   : entry_o(eh);
+                            const int f_h = t + op_h - 1, a_h = l - t + 1;
+                            bool ok = true;
+                            long long S = 0;
+                            for (int base = 0; base < nP; base += 32) {
+                                const int i = base + lane;
+                                const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
+                                if (swi != kDead) {
+                                    const uint64_t ei = RING(WR(head + i));
+                                    int f_i = (int)swi;
+                                    if (worst) f_i += p.tables[1 + p.n_classes + entry_cls(ei)].vmin +
+                                                      (int)p.tables[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
+                                    const int a_i = entry_l(ei) + entry_o(ei) - (int)swi;
+                                    if (f_i <= f_h && (long long)vproj[WA(shead + i)] + a_h + f_i > M) ok = false;
+                                    if (f_i >= f_h) S += a_i + f_h;
+                                }
+                            }
+                            S = warp_sum64(S) + a_h + f_h;
+                            if (__any_sync(FULL, !ok) || S > M) { CADD(C_GATE_BLOCKED, 1); break; }
+                            for (int base = 0; base < nP; base += 32) {   // it starts: it adds to every earlier last slot
+                                const int i = base + lane;
+                                const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
+                                if (swi != kDead) {
+                                    int f_i = (int)swi;
+                                    if (worst) {
+                                        const uint64_t ei = RING(WR(head + i));
+                                        f_i += p.tables[1 + p.n_classes + entry_cls(ei)].vmin +
+                                               (int)p.tables[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
+                                    }
+                                    if (f_i <= f_h) vproj[WA(shead + i)] += a_h + f_i;
+                                }
+                            }
+                            if (lane == 0) vproj[WA(shead + nP)] = (int)S;
+                        }
                         uint32_t sw;
                         if (g == l) {
                             sw = (uint32_t)(t + entry_o(RING(WR(head + nP))) - 1);
@@ -671,7 +724,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             Ndec--;
                         }
                         q_l = entry_l(e);
-                        if ((kClassFlow && policy == 4) && lane == 0) qcnt[entry_cls(e)] += 1;
+                        if ((kExt && policy == 4) && lane == 0) qcnt[entry_cls(e)] += 1;
                         nP--;
                         nQ++;
                         nev++;
@@ -704,9 +757,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
                             const bool done = (sw == (uint32_t)t);
                             const uint32_t m = __ballot_sync(FULL, done);
+                            uint64_t e = 0;
                             if (m) {
                                 if (done) {
-                                    const uint64_t e = RING(WR(head + i));
+                                    e = RING(WR(head + i));
                                     const int l = entry_l(e), o = entry_o(e);
                                     const int lat = t - entry_tarr(e) + 1;
                                     acc_lat += (unsigned)lat;
@@ -722,6 +776,30 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     STATE(WA(shead + i)) = kDead;
                                 }
                                 ndone += __popc(m);
+                                if (kExt && policy == 5 && grp.mc_worst != 0) {
+                                    // MC benchmark with worst-case projection: a request that ends before its
+                                    // projected last slot f_c leaves the projected usage of every last slot <= f_c
+                                    __syncwarp();
+                                    uint32_t fm = m;
+                                    while (fm) {
+                                        const int src = __ffs(fm) - 1;
+                                        fm &= fm - 1;
+                                        const uint64_t ec = __shfl_sync(FULL, e, src);
+                                        const DevTable dc = p.tables[1 + p.n_classes + entry_cls(ec)];
+                                        const int f_c = t - entry_o(ec) + dc.vmin + (int)dc.n - 1;
+                                        const int a_c = entry_l(ec) + entry_o(ec) - t;
+                                        for (int vb = 0; vb < nP; vb += 32) {
+                                            const int vi = vb + lane;
+                                            const uint32_t swv = (vi < nP) ? STATE(WA(shead + vi)) : kDead;
+                                            if (swv != kDead) {
+                                                const uint64_t ev = RING(WR(head + vi));
+                                                const DevTable dv = p.tables[1 + p.n_classes + entry_cls(ev)];
+                                                const int f_v = (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev);
+                                                if (f_v <= f_c) vproj[WA(shead + vi)] -= a_c + f_v;
+                                            }
+                                        }
+                                    }
+                                }
                             }
                             gmin = min(gmin, __reduce_min_sync(FULL, (done || sw == kDead) ? kNoFin : sw));
                         }

@@ -325,8 +325,9 @@ def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2) -> SimConf
     """The paper's own synthetic setting (Section 4.1): three classes (l, o) = (10,20), (10,40), (10,60),
     Poisson arrivals of total intensity 5 per slot split evenly over the classes, M = 16492, no token
     budget, T up to 10000.  Policies on common random numbers: Algorithm 2 with b = 12 (the sum of the
-    paper's per-class budgets 4+4+4), greedy, alpha-protection greedy, and Algorithm 1 with the paper's
-    budgets (4, 4, 4), for which sum_k b_k w_k = 16240 < M (Eq. 2)."""
+    paper's per-class budgets 4+4+4), greedy, alpha-protection greedy, Algorithm 1 with the paper's
+    budgets (4, 4, 4), for which sum_k b_k w_k = 16240 < M (Eq. 2), and the MC benchmark with known and with
+    worst-case output lengths."""
     class_law = Table(0, np.array([1431655765, 2863311530, 0xFFFFFFFF], dtype=np.uint32))
     prompt = tuple(constant_table(10) for _ in range(3))
     decode = tuple(constant_table(o) for o in (20, 40, 60))
@@ -337,7 +338,9 @@ def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2) -> SimConf
         groups=(Group(POLICY_FLOW, b_fp=12 << 16, n_replicas=replicas),
                 Group(POLICY_GREEDY, n_replicas=replicas),
                 Group(POLICY_ALPHA, n_replicas=replicas, m_admit=int(math.floor((1.0 - alpha) * M))),
-                Group(POLICY_CLASSFLOW, n_replicas=replicas, b_class=(4, 4, 4))),
+                Group(POLICY_CLASSFLOW, n_replicas=replicas, b_class=(4, 4, 4)),
+                Group(POLICY_MC, n_replicas=replicas, mc_worst_case=0),
+                Group(POLICY_MC, n_replicas=replicas, mc_worst_case=1)),
         trace_stride=1, hist_bins=1024, hist_shift=0, complog_cap=0, name="cfg6-paper-section-4.1")
 
 

@@ -128,6 +128,10 @@ def test_config6_full_paper_setting():
     n = cfg.groups[0].n_replicas
     assert c[:n, I["overflow_steps"]].sum() == 0 and c[:, I["dropped"]].sum() == 0
     # Algorithm 1 with b = (4,4,4) (last group): usage never passes sum_k b_k w_k = 16240 < M, no eviction (Thm. 3.3)
-    alg1 = c[3 * n:]
+    alg1 = c[3 * n:4 * n]
     assert (alg1[:, I["max_U"]] <= 16240).all() and alg1[:, I["evictions"]].sum() == 0
     assert alg1[:, I["gate_blocked_steps"]].sum() == 0 and alg1[:, I["completed"]].min() > 40000
+    # MC benchmark (known and worst-case lengths): admissions are proved to fit, so nothing is ever evicted
+    mc = c[4 * n:]
+    assert mc[:, I["evictions"]].sum() == 0 and mc[:, I["overflow_steps"]].sum() == 0
+    assert mc[:, I["completed"]].min() > 40000
