@@ -321,20 +321,22 @@ def config5(replicas: int = 131072, T: int = 100000) -> SimConfig:
         trace_stride=0, hist_bins=1024, hist_shift=7, complog_cap=0, name="cfg5-large-bursty")
 
 
-def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2) -> SimConfig:
+def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2, total_rate: float = 5.0) -> SimConfig:
     """The paper's own synthetic setting (Section 4.1): three classes (l, o) = (10,20), (10,40), (10,60),
     Poisson arrivals of total intensity 5 per slot split evenly over the classes, M = 16492, no token
     budget, T up to 10000.  Policies on common random numbers: Algorithm 2 with b = 12 (the sum of the
     paper's per-class budgets 4+4+4), greedy, alpha-protection greedy, Algorithm 1 with the paper's
     budgets (4, 4, 4), for which sum_k b_k w_k = 16240 < M (Eq. 2), and the MC benchmark with known and with
-    worst-case output lengths."""
+    worst-case output lengths.  ``total_rate`` = 5 reads the paper's "intensity 5" as the total rate (load
+    0.41 of capacity); 15 reads it as 5 per class (load 1.23: memory binds and the policies separate, but the
+    finite waiting room then drops arrivals, which the paper's unbounded queue does not)."""
     class_law = Table(0, np.array([1431655765, 2863311530, 0xFFFFFFFF], dtype=np.uint32))
     prompt = tuple(constant_table(10) for _ in range(3))
     decode = tuple(constant_table(o) for o in (20, 40, 60))
     M = 16492
     return SimConfig(
         M=M, K=0, T_max=T, Qcap=256, Acap=1024, seed=6, class_law=class_law, prompt=prompt, decode=decode,
-        arrivals=(Arrivals((poisson_table(5.0),)),),
+        arrivals=(Arrivals((poisson_table(total_rate),)),),
         groups=(Group(POLICY_FLOW, b_fp=12 << 16, n_replicas=replicas),
                 Group(POLICY_GREEDY, n_replicas=replicas),
                 Group(POLICY_ALPHA, n_replicas=replicas, m_admit=int(math.floor((1.0 - alpha) * M))),
