@@ -260,22 +260,29 @@ def main():
     # end to end through the host-buffer entry point: tables from host memory, every output back to host
     e2e = None
     out_bytes = sizes["counters"] + sizes["trace"] + sizes["hist"] + sizes["complog"]
-    if rank == 0 and world == 1 and not args.no_e2e and out_bytes > 8e9:
+    if not args.no_e2e and out_bytes > 8e9:
         e2e = {"value": None, "unit": UNIT,
                "skipped": "outputs of %.1f GB are not copied to host buffers in the default run" % (out_bytes / 1e9)}
-    elif rank == 0 and world == 1 and not args.no_e2e:
-        torch.cuda.synchronize()
+    elif not args.no_e2e:
+        # every rank runs its own shard through the host-buffer entry point; the time is the maximum over ranks
+        barrier()
         t0 = time.perf_counter()
         out = fb.fcsim_simulate_host(cfg, total_steps)
         dt = time.perf_counter() - t0
         assert (out["counters"] == counters).all(), "host-buffer run differs from the device-buffer run"
+        if dist is not None:
+            tm = torch.tensor([dt], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            dt = float(tm.item())
         table_bytes = 4 * (cfg.class_law.n + sum(t.n for t in cfg.prompt) + sum(t.n for t in cfg.decode)
                            + sum(t.n for a in cfg.arrivals for t in a.count))
         n_all = args.warmup + args.steps
-        e2e = {"value": R * total_steps / dt, "unit": UNIT,
-               "h2d_bytes_per_step": table_bytes / n_all, "d2h_bytes_per_step": (out_bytes + sizes["scratch"]) / n_all,
+        e2e = {"value": world * R * total_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": world * table_bytes / n_all,
+               "d2h_bytes_per_step": world * (out_bytes + sizes["scratch"]) / n_all,
                "what": "fcsim_simulate_host: tables H2D + all %d slots from the empty system + every output "
-                       "copied to host buffers, wall clock; bytes amortised over %d steps" % (total_steps, n_all),
+                       "copied to host buffers, wall clock (max over ranks); bytes amortised over %d steps"
+                       % (total_steps, n_all),
                "seconds": round(dt, 3)}
 
     if rank != 0:
