@@ -267,16 +267,32 @@ def fcsim_strerror(code: int) -> str:
     return load().fcsim_strerror(int(code)).decode()
 
 
-def fcsim_simulate_host(cfg, n_steps: Optional[int] = None, trace=True, hist=True, complog=True) -> dict:
-    """Whole job with host (numpy) outputs; device memory is managed inside the library."""
+def host_output_arrays(cfg, trace=True, hist=True, complog=True, pinned=False) -> dict:
+    """Host arrays shaped for fcsim_simulate_host; ``pinned`` takes page-locked memory from torch."""
+    R = cfg.n_replicas
+    n_rec = cfg.T_max // cfg.trace_stride if cfg.trace_stride > 0 else 0
+
+    def alloc(shape, dtype):
+        if not pinned:
+            return np.zeros(shape, dtype=dtype)
+        import torch
+        tdt = {np.int32: torch.int32, np.int64: torch.int64}[dtype]
+        return torch.zeros(shape, dtype=tdt, pin_memory=True).numpy()
+    return {"counters": alloc((R, N_COUNTERS), np.int64),
+            "trace": alloc((R, n_rec, 2), np.int32) if (trace and n_rec) else None,
+            "hist": alloc((R, cfg.hist_bins), np.int32) if (hist and cfg.hist_bins) else None,
+            "complog": alloc((R, cfg.complog_cap, 2), np.int32) if (complog and cfg.complog_cap) else None}
+
+
+def fcsim_simulate_host(cfg, n_steps: Optional[int] = None, trace=True, hist=True, complog=True,
+                        out: Optional[dict] = None) -> dict:
+    """Whole job with host (numpy) outputs; device memory is managed inside the library.
+    ``out``: arrays from host_output_arrays to fill (allocated here when None)."""
     c, keep = marshal_config(cfg)
     n_steps = cfg.T_max if n_steps is None else int(n_steps)
-    R, G = cfg.n_replicas, len(cfg.groups)
-    n_rec = cfg.T_max // cfg.trace_stride if cfg.trace_stride > 0 else 0
-    out = {"counters": np.zeros((R, N_COUNTERS), dtype=np.int64)}
-    out["trace"] = np.zeros((R, n_rec, 2), dtype=np.int32) if (trace and n_rec) else None
-    out["hist"] = np.zeros((R, cfg.hist_bins), dtype=np.int32) if (hist and cfg.hist_bins) else None
-    out["complog"] = np.zeros((R, cfg.complog_cap, 2), dtype=np.int32) if (complog and cfg.complog_cap) else None
+    G = len(cfg.groups)
+    if out is None:
+        out = host_output_arrays(cfg, trace, hist, complog)
     summ = (fcsim_summary * G)()
 
     def ptr(a):
