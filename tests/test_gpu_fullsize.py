@@ -135,3 +135,13 @@ def test_config6_full_paper_setting():
     mc = c[4 * n:]
     assert mc[:, I["evictions"]].sum() == 0 and mc[:, I["overflow_steps"]].sum() == 0
     assert mc[:, I["completed"]].min() > 40000
+
+
+def test_one_call_split_into_several_launches():
+    # 262 144 replicas: the library splits a 10 000-slot call into launches of at most 8 192 slots
+    from paper_2604_11001_b200 import binding as fb
+    cfg = wl.config5(T=10000)
+    sim = fb.Simulation(cfg)
+    assert sim.launch_info()["max_steps_per_launch"] < 10000
+    sim.close()
+    _run_full(cfg, 10000, list(range(5, cfg.n_replicas, 16411)))
