@@ -381,6 +381,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         while (t < t_end) {
             // -------------------------------------------------------------- batch: draws of up to 32 slots
             int L = min(32, t_end - t);
+            __syncwarp();  // the staged arrivals of the previous batch have all been read
             uint32_t w0, w1, w2, w3;
             philox4x32_10((uint32_t)(t + 1 + lane), rid, 0u, 0u, p.key0, p.key1, w0, w1, w2, w3);
             const int Bt = (int)(grp.b_fp >> 16) + (((w1 >> 16) < (grp.b_fp & 0xffffu)) ? 1 : 0);
@@ -514,7 +515,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 int a = 0;
                 const int cap = (policy == 0) ? B_t : 0x7fffffff;
                 for (;;) {
-                    if (squeeze) { compact(); rebuild_minima(); squeeze = false; }
+                    if (squeeze) {
+                        __syncwarp();  // state words written by lane 0 during this slot's activations
+                        compact();
+                        rebuild_minima();
+                        squeeze = false;
+                    }
                     if ((kExt && policy == 4)) {
                         // Algorithm 1: for every class k, up to b_k waiting requests of that class, oldest first.
                         // The pick leaves the middle of the queue: the entries ahead of it move one place
@@ -650,6 +656,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             n_pref++;
                         }
                         if (lane == 0) STATE(WA(shead + nP)) = sw;
+                        __syncwarp();  // the next pick may scan the active range (MC projection) or squeeze it
                         nP++;
                         nQ--;
                         q_l = -1;
@@ -917,6 +924,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             default: break;
         }
         if (lane < kHeaderWords) hdr[lane] = out;
+        __syncwarp();  // every lane's last writes to the rings are visible before they are copied out
         {
             uint4* dst = reinterpret_cast<uint4*>(ws + kHeaderWords * 4);
             const uint4* src = reinterpret_cast<const uint4*>(my);
