@@ -255,6 +255,7 @@ struct fcsim {
     uint32_t* d_pool = nullptr;
     unsigned short* d_gpool = nullptr;
     int32_t* d_bclass = nullptr;
+    size_t tabcache_off = 0, smem_block = 0;
     void (*kernel)(const Params) = nullptr;  // step kernel variant for this configuration
     DevTable* d_tables = nullptr;
     DevArrivals* d_arrivals = nullptr;
@@ -296,8 +297,9 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         pool.insert(pool.end(), t.cdf, t.cdf + t.n);
         if (t.n >= 16) {
             // guide[b] = first k < n-1 with cdf[k] > (b << shift), else n-1; guide[2^bits] = n-1
+            // about two table entries per bucket, so that the search after the guide is one or two probes
             uint32_t bits = 4;
-            while (bits < 10 && (4u << bits) < t.n) ++bits;
+            while (bits < 12 && (2u << bits) < t.n) ++bits;
             const uint32_t shift = 32 - bits;
             d.guide = (bits << 27) | (uint32_t)gpool.size();
             uint32_t k = 0;
@@ -413,8 +415,20 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     rc = upload_tables(h, cfg);
     if (rc != FCSIM_OK) return fail(rc);
 
-    const size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
+    size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
     if (smem_block > (size_t)prop.sharedMemPerBlockOptin) return fail(FCSIM_ECAP);
+    {   // a copy of the table descriptors behind the warps' slices, if it does not cost a resident CTA
+        const size_t extra = align_up((size_t)(1 + 2 * cfg->n_classes) * sizeof(DevTable), 16);
+        const size_t sm = (size_t)prop.sharedMemPerMultiprocessor;
+        auto ctas = [&](size_t b) { return sm / (align_up(b, 1024) + 1024); };
+        h->tabcache_off = 0;
+        if (cfg->n_classes <= 16 && smem_block + extra <= (size_t)prop.sharedMemPerBlockOptin &&
+            ctas(smem_block + extra) == ctas(smem_block)) {
+            h->tabcache_off = smem_block;
+            smem_block += extra;
+        }
+    }
+    h->smem_block = smem_block;
     // six CTAs per SM need <= 80 registers per thread and their shared memory (plus 1 KB each that the
     // system reserves) within the SM's 228 KB; otherwise the 5-CTA register allocation is the better one
     const bool six = 6 * (smem_block + 1024) <= (size_t)prop.sharedMemPerMultiprocessor;
@@ -458,6 +472,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.qcnt_off = (uint32_t)L.qcnt_off;
     p.tstage_off = (uint32_t)L.tstage_off;
     p.state_bytes = (uint32_t)L.state_bytes;
+    p.tabcache_off = (uint32_t)h->tabcache_off;
     p.has_v = L.has_v;
     p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
     p.workspace = static_cast<unsigned char*>(b->workspace);
@@ -484,7 +499,7 @@ extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
     if ((long long)h->t_done + n_steps > h->cfg.T_max) return FCSIM_ERANGE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int per = max_steps_per_launch(h);
-    const size_t smem_block = (size_t)h->L.warps_per_block * h->L.smem_per_warp;
+    const size_t smem_block = h->smem_block;
     int left = n_steps;
     while (left > 0) {
         const int now = std::min(left, per);
@@ -643,7 +658,7 @@ extern "C" int fcsim_get_launch_info(const fcsim_t* h, fcsim_launch_info* out) {
     out->warps_per_block = h->L.warps_per_block;
     out->blocks_per_sm = h->blocks_per_sm;
     out->sm_count = h->sm_count;
-    out->smem_per_block = (int32_t)(h->L.warps_per_block * h->L.smem_per_warp);
+    out->smem_per_block = (int32_t)h->smem_block;
     out->smem_per_warp = (int32_t)h->L.smem_per_warp;
     out->max_steps_per_launch = max_steps_per_launch(h);
     return FCSIM_OK;

@@ -73,6 +73,7 @@ struct Params {
     const unsigned short* gpool;  // guide tables: for bucket b of the top bits of u, the first candidate index
     const int32_t* bclass;        // per-class budgets b_k of the Algorithm-1 groups
     uint32_t qcnt_off;            // byte offset of the per-class queue counts in a warp's shared memory (0 = none)
+    uint32_t tabcache_off;        // byte offset in the CTA's shared memory of a copy of `tables` (0 = none)
     uint32_t state_bytes;         // ring + state words (+ projection words): what is saved between launches
     int32_t has_v;                // 1 = a projection word per active entry follows the state words (MC benchmark)
     uint32_t tstage_off;          // byte offset of the trace staging area (2 x 32 records) in a warp's shared
@@ -143,6 +144,37 @@ __device__ __forceinline__ void bulk_wait_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Two independent table searches (prompt and decode length of one arrival) advanced in the same loop, so
+// that their dependent global loads overlap instead of running one chain after the other.
+__device__ __forceinline__ void sample_pair(const uint32_t* __restrict__ pool, const unsigned short* __restrict__ gpool,
+                                            const DevTable ta, uint32_t ua, const DevTable tb, uint32_t ub, int& va,
+                                            int& vb) {
+    const uint32_t* __restrict__ ca = pool + ta.off;
+    const uint32_t* __restrict__ cb = pool + tb.off;
+    uint32_t loa = 0, hia = ta.n - 1, lob = 0, hib = tb.n - 1;
+    const uint32_t ga = ta.guide >> 27, gb = tb.guide >> 27;
+    if (ga) {
+        const unsigned short* __restrict__ g = gpool + (ta.guide & 0x7ffffffu);
+        const uint32_t b = ua >> (32u - ga);
+        loa = __ldg(g + b);
+        hia = __ldg(g + b + 1);
+    }
+    if (gb) {
+        const unsigned short* __restrict__ g = gpool + (tb.guide & 0x7ffffffu);
+        const uint32_t b = ub >> (32u - gb);
+        lob = __ldg(g + b);
+        hib = __ldg(g + b + 1);
+    }
+    while (loa < hia || lob < hib) {
+        const uint32_t ma = (loa + hia) >> 1, mb = (lob + hib) >> 1;
+        const uint32_t xa = __ldg(ca + ma), xb = __ldg(cb + mb);  // both probes in flight together (in range always)
+        if (loa < hia) { if (xa > ua) hia = ma; else loa = ma + 1; }
+        if (lob < hib) { if (xb > ub) hib = mb; else lob = mb + 1; }
+    }
+    va = ta.vmin + (int)loa;
+    vb = tb.vmin + (int)lob;
+}
 
 __device__ __forceinline__ uint32_t lanemask_lt() {
     uint32_t m;
@@ -217,6 +249,15 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 template <bool kExt, int kMinCtas>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    // the table descriptors of the length laws are read for every generated arrival: the host reserves room
+    // for a copy behind the warps' slices when that does not cost a resident CTA
+    const bool tab_shared = p.tabcache_off != 0;
+    DevTable* s_tables = reinterpret_cast<DevTable*>(smem_raw + p.tabcache_off);
+    if (tab_shared) {
+        for (int i = threadIdx.x; i < 1 + 2 * p.n_classes; i += blockDim.x) s_tables[i] = p.tables[i];
+    }
+    __syncthreads();
+    const DevTable* __restrict__ tabs = tab_shared ? s_tables : p.tables;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     unsigned char* my = smem_raw + (size_t)warp * p.smem_per_warp;
@@ -425,9 +466,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     uint32_t a0, a1, a2, a3;
                     philox4x32_10((uint32_t)(t + 1 + lo), rid, 1u, (uint32_t)(idx - ex_k), p.key0, p.key1, a0, a1,
                                   a2, a3);
-                    const int cls = sample_table(p.pool, p.gpool, p.tables[0], a0);
-                    const int l = sample_table(p.pool, p.gpool, p.tables[1 + cls], a1);
-                    const int o = sample_table(p.pool, p.gpool, p.tables[1 + p.n_classes + cls], a2);
+                    const int cls = sample_table(p.pool, p.gpool, tabs[0], a0);
+                    int l, o;
+                    sample_pair(p.pool, p.gpool, tabs[1 + cls], a1, tabs[1 + p.n_classes + cls], a2, l, o);
                     STAGE(idx) = pack_entry(l, o, t + 1 + lo, cls);
                 }
             }
