@@ -390,3 +390,31 @@ def random_small_config(seed: int, n_replicas: int = 4, T: int = 60) -> SimConfi
         arrivals=tuple(arrivals), groups=tuple(groups), trace_stride=stride,
         hist_bins=int(rng.choice([0, 8, 16])), hist_shift=int(rng.integers(0, 3)),
         complog_cap=int(rng.choice([0, 5, 64])), name=f"random-{seed}")
+
+
+def random_medium_config(seed: int, n_replicas: int = 2) -> SimConfig:
+    """A seeded, randomly parameterised simulation on the length laws of presets 2, 4 or 5 with a few
+    thousand slots: three random policies, random capacities, budget, arrival law and outputs."""
+    rng = np.random.default_rng(10_000 + seed)
+    base = (config5, config2, config4)[int(rng.integers(0, 3))](replicas=1, T=100)
+    T = int(rng.integers(1500, 4000))
+    lmax = max(t.vmax for t in base.prompt)
+    omax = max(t.vmax for t in base.decode)
+    M = int(rng.integers(lmax + omax, 6 * (lmax + omax)))
+    groups = []
+    for pol in rng.permutation(6)[:3]:
+        groups.append(Group(int(pol), b_fp=int(rng.integers(0, 4 * 65536)), chunk=int(rng.choice([64, 512, 3000])),
+                            arrivals_id=0, rng_replica_base=int(rng.integers(0, 1000)), n_replicas=n_replicas,
+                            m_admit=int(rng.integers(M // 2, M + 1)),
+                            b_class=tuple(int(x) for x in rng.integers(0, 3, size=base.n_classes)),
+                            mc_worst_case=int(rng.integers(0, 2))))
+    lam = float(rng.uniform(0.2, 4.0))
+    if rng.random() < 0.6:
+        arr = Arrivals((poisson_table(lam),))
+    else:
+        arr = Arrivals((poisson_table(lam * 0.3), poisson_table(lam * 1.5)),
+                       (int(rng.integers(0, 2 ** 28)), int(rng.integers(0, 2 ** 28))))
+    return base.with_(M=M, K=int(rng.choice([0, 0, 700, 2048])), T_max=T, Qcap=int(rng.choice([8, 40, 256])),
+                      Acap=int(rng.choice([48, 96, 200, 512])), seed=int(rng.integers(0, 2 ** 62)), arrivals=(arr,),
+                      groups=tuple(groups), trace_stride=int(rng.choice([1, 1, 5])), hist_bins=64, hist_shift=6,
+                      complog_cap=int(rng.choice([0, 300, 20000])), name=f"medium-{seed}")

@@ -181,3 +181,13 @@ def test_horizon_limit_and_range_errors():
     # slots close to the 24-bit horizon limit: arrival times near 2^24 must survive the packing
     late = wl.config1(replicas=2, T=(1 << 24) - 1)
     assert fb.fcsim_query_sizes(late.with_(trace_stride=0, complog_cap=0))["trace"] == 0
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_medium_configs(seed):
+    # preset-sized laws, thousands of slots, every policy: lazy removal, in-place eviction, storage-bound
+    # squeezes and resumed launches all occur
+    cfg = wl.random_medium_config(seed)
+    cut = 1 + (seed * 97) % (cfg.T_max - 1)
+    ref = orc.run(cfg, threads=4)
+    assert_same(cfg, run_gpu(cfg, pieces=[cut, cfg.T_max - cut]), ref, cfg.T_max, cfg.name)

@@ -72,6 +72,16 @@ def test_identities_on_random_tiny_configs(seed):
     check_identities(cfg, out, cfg.T_max)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_identities_on_random_medium_configs(seed):
+    cfg = wl.random_medium_config(seed)
+    out = orc.run(cfg, threads=4)
+    c = out["counters"].astype(object)
+    assert (c[:, I["arrived"]] == c[:, I["dropped"]] + c[:, I["completed"]] + c[:, I["q_final"]] + c[:, I["p_final"]]).all()
+    assert (c[:, I["sum_N"]] == c[:, I["sum_lat"]] + c[:, I["resid_age"]]).all()
+    assert (c[:, I["max_U"]] <= cfg.M).all()
+
+
 def test_pause_point_extras_are_a_prefix_property():
     # counters of a run stopped after a slots equal a run of a slots: the model is causal
     cfg = wl.config1(replicas=4, T=600)
