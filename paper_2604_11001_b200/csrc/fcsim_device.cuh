@@ -1,5 +1,6 @@
-// Device side of fcsim: one warp advances one replica of the serving model of Section 2.1
-// under Algorithm 2 (or the greedy / chunked-prefill baselines), slot by slot.
+// Device side of fcsim: one warp advances one replica of the serving model of Section 2.1, slot by slot,
+// under Algorithm 2, Algorithm 1, or one of the baselines (greedy, chunked prefill, alpha-protection greedy,
+// MC benchmark).
 //
 // Data layout per replica (shared memory while a warp owns the replica, the same bytes in the
 // caller's workspace between launches):
@@ -16,7 +17,12 @@
 //                      prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so far;
 //                      0 for a request that has completed but whose entry has not been squeezed
 //                      out yet (completed entries are removed lazily, many at a time).
+//                      Under Algorithm 1 a pick may leave the middle of the queue (first request of a
+//                      class); the entries ahead of it then shift by one place.
+//   vproj [Acap] i32   only with MC groups: projected memory usage of the last slot of each active entry.
 //   stage [S]    u64   arrivals generated ahead of time for the next batch of <= 32 slots.
+//   qcnt  [classes] u32  only with Algorithm-1 groups: waiting requests per class.
+// Only ring, state and vproj are saved between launches (plus 16 scalar words); the rest is rebuilt.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
