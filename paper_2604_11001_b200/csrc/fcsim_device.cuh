@@ -347,7 +347,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         uint32_t sumN = 0, tokgen = 0, arrived = 0, dropped = 0;
         int maxU = 0, maxQ = 0;
         int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
-        int q_l = -1;  // prompt length of the queue head when known (saves a shared-memory read per blocked slot)
+        uint64_t q_e = 0;  // the queue head's entry when known, else 0 (saves shared-memory reads in blocked slots)
         // statistics of completions, private to the lane that saw them; reduced once when the replica is put back
         unsigned long long acc_lat = 0, acc_w = 0;
         uint32_t acc_o = 0, completed = 0;
@@ -625,7 +625,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         if (gate_hit) CADD(C_GATE_BLOCKED, 1);
                         if (budget_hit) CADD(C_BUDGET_BLOCKED, 1);
                         if (storage_hit) { CADD(C_ACAP_BLOCKED, 1); status |= 1u; }
-                        q_l = -1;
+                        q_e = 0;
                         break;
                     }
                     while (a < cap && nQ > 0) {
@@ -633,8 +633,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room
                             CADD(C_ACAP_BLOCKED, 1); status |= 1u; break;
                         }
-                        if (q_l < 0) q_l = entry_l(RING(WR(head + nP)));
-                        const int l = q_l;
+                        if (q_e == 0) q_e = RING(WR(head + nP));
+                        const int l = entry_l(q_e);
                         int g, need;
                         if (policy == 2) {
                             g = kinf ? min(chunk, l) : min(min(chunk, l), R);
@@ -653,7 +653,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             // vproj[k] holds the usage of slot f_k for the running requests, so the head h
                             // (last slot f_h) fits iff vproj[k] + a_h + f_k <= M for every k with f_k <= f_h and
                             // the usage of slot f_h itself, sum over f_i >= f_h of (a_i + f_h) + a_h + f_h, is <= M.
-                            const uint64_t eh = RING(WR(head + nP));
+                            const uint64_t eh = q_e;
                             const bool worst = grp.mc_worst != 0;
                             const int op_h = worst ? (p.tables[1 + p.n_classes + entry_cls(eh)].vmin +
                                                       (int)p.tables[1 + p.n_classes + entry_cls(eh)].n - 1)
@@ -693,7 +693,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         }
                         uint32_t sw;
                         if (g == l) {
-                            sw = (uint32_t)(t + entry_o(RING(WR(head + nP))) - 1);
+                            sw = (uint32_t)(t + entry_o(q_e) - 1);
                             next_fin = min(next_fin, sw);
                             if (lane == (nP >> bsh)) cmin = min(cmin, sw);
                             Ndec++;
@@ -706,7 +706,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         __syncwarp();  // the next pick may scan the active range (MC projection) or squeeze it
                         nP++;
                         nQ--;
-                        q_l = -1;
+                        q_e = 0;
                         G += need;
                         if (!kinf) R -= min(g, R);
                         a++;
@@ -739,7 +739,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         Ndec = 0;
                         n_pref = 0;
                         G = 0;
-                        q_l = -1;
+                        q_e = 0;
                         cmin = kNoFin;
                         next_fin = kNoFin;
                     }
@@ -777,7 +777,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             wasted += j;
                             Ndec--;
                         }
-                        q_l = entry_l(e);
+                        q_e = e;
                         if ((kExt && policy == 4) && lane == 0) qcnt[entry_cls(e)] += 1;
                         nP--;
                         nQ++;
