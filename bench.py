@@ -31,7 +31,7 @@ UNIT = "replica-steps/s"
 # Executed warp-instructions per replica-step of the step kernel in the timed regime of each preset,
 # from the committed ncu captures (profiles/): smsp__inst_executed.sum / (replicas x slots) of one launch.
 # None = not captured for the current kernel.
-INST_PER_REPLICA_STEP = {1: None, 2: None, 3: 361.7, 4: None, 5: 264.6, 6: None}
+INST_PER_REPLICA_STEP = {1: None, 2: None, 3: 352.9, 4: None, 5: 260.4, 6: None}
 # DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
 DRAM_BYTES_PER_REPLICA_STEP = {1: None, 2: None, 3: 17.8, 4: None, 5: 7.9, 6: None}
 
