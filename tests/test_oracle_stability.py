@@ -51,3 +51,22 @@ def test_underloaded_flow_control_stays_bounded_without_overflow():
     L = c[I["sum_N"]] / (cfg.n_replicas * 2 * T)
     W = c[I["sum_lat"]] / c[I["completed"]]
     assert abs(L - lam * W) / L < 0.02
+
+
+def test_overflow_count_respects_the_bound_of_theorem_3_6():
+    # Thm. 3.6: b E[w] <= (1 - eps) M, B_t <= A, lengths <= C  =>  E[#overflow slots] < T exp(-eps^2 M^2 / (2 (A^2+A) C^3)).
+    # The bound is loose at these sizes (close to T); the slots in which memory binds (an eviction, or an
+    # activation refused by the headroom gate) must stay below it -- here they are in fact zero.
+    import math
+    T = 20000
+    cfg, ew, lam = _cfg(0.6, 0.8, T)
+    b = cfg.groups[0].b_fp / 65536.0
+    eps = 1.0 - b * ew / cfg.M
+    assert eps > 0.19
+    A = int(b) + 1
+    C = 512
+    bound = T * math.exp(-(eps * cfg.M) ** 2 / (2.0 * (A * A + A) * C ** 3))
+    out = orc.run(cfg, threads=6)
+    binding = (out["counters"][:, I["overflow_steps"]] + out["counters"][:, I["gate_blocked_steps"]]).mean()
+    assert binding < bound
+    assert binding == 0
