@@ -655,8 +655,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             // the usage of slot f_h itself, sum over f_i >= f_h of (a_i + f_h) + a_h + f_h, is <= M.
                             const uint64_t eh = q_e;
                             const bool worst = grp.mc_worst != 0;
-                            const int op_h = worst ? (p.tables[1 + p.n_classes + entry_cls(eh)].vmin +
-                                                      (int)p.tables[1 + p.n_classes + entry_cls(eh)].n - 1)
+                            const int op_h = worst ? (tabs[1 + p.n_classes + entry_cls(eh)].vmin +
+                                                      (int)tabs[1 + p.n_classes + entry_cls(eh)].n - 1)
                                                    : entry_o(eh);
                             const int f_h = t + op_h - 1, a_h = l - t + 1;
                             bool ok = true;
@@ -667,8 +667,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 if (swi != kDead) {
                                     const uint64_t ei = RING(WR(head + i));
                                     int f_i = (int)swi;
-                                    if (worst) f_i += p.tables[1 + p.n_classes + entry_cls(ei)].vmin +
-                                                      (int)p.tables[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
+                                    if (worst) f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
+                                                      (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
                                     const int a_i = entry_l(ei) + entry_o(ei) - (int)swi;
                                     if (f_i <= f_h && (long long)vproj[WA(shead + i)] + a_h + f_i > M) ok = false;
                                     if (f_i >= f_h) S += a_i + f_h;
@@ -683,8 +683,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     int f_i = (int)swi;
                                     if (worst) {
                                         const uint64_t ei = RING(WR(head + i));
-                                        f_i += p.tables[1 + p.n_classes + entry_cls(ei)].vmin +
-                                               (int)p.tables[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
+                                        f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
+                                               (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
                                     }
                                     if (f_i <= f_h) vproj[WA(shead + i)] += a_h + f_i;
                                 }
@@ -839,7 +839,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                         const int src = __ffs(fm) - 1;
                                         fm &= fm - 1;
                                         const uint64_t ec = __shfl_sync(FULL, e, src);
-                                        const DevTable dc = p.tables[1 + p.n_classes + entry_cls(ec)];
+                                        const DevTable dc = tabs[1 + p.n_classes + entry_cls(ec)];
                                         const int f_c = t - entry_o(ec) + dc.vmin + (int)dc.n - 1;
                                         const int a_c = entry_l(ec) + entry_o(ec) - t;
                                         for (int vb = 0; vb < nP; vb += 32) {
@@ -847,7 +847,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                             const uint32_t swv = (vi < nP) ? STATE(WA(shead + vi)) : kDead;
                                             if (swv != kDead) {
                                                 const uint64_t ev = RING(WR(head + vi));
-                                                const DevTable dv = p.tables[1 + p.n_classes + entry_cls(ev)];
+                                                const DevTable dv = tabs[1 + p.n_classes + entry_cls(ev)];
                                                 const int f_v = (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev);
                                                 if (f_v <= f_c) vproj[WA(shead + vi)] -= a_c + f_v;
                                             }
