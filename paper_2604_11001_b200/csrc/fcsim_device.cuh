@@ -348,6 +348,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         int maxU = 0, maxQ = 0;
         int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
         uint64_t q_e = 0;  // the queue head's entry when known, else 0 (saves shared-memory reads in blocked slots)
+        // Whole-prompt policies: once the headroom gate has refused the queue head, it keeps refusing it until
+        // memory is released (a completion or an eviction): the usage only grows and the head does not change.
+        // While the flag is up a slot's activation attempt is just counted as refused.
+        bool gate_closed = false;
         // statistics of completions, private to the lane that saw them; reduced once when the replica is put back
         unsigned long long acc_lat = 0, acc_w = 0;
         uint32_t acc_o = 0, completed = 0;
@@ -561,6 +565,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
                 int a = 0;
                 const int cap = (policy == 0) ? B_t : 0x7fffffff;
+                if (gate_closed && !squeeze) {
+                    if (cap > 0) CADD(C_GATE_BLOCKED, 1);
+                } else
                 for (;;) {
                     if (squeeze) {
                         __syncwarp();  // state words written by lane 0 during this slot's activations
@@ -645,7 +652,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             if (!(kinf || a == 0 || g <= R)) { CADD(C_BUDGET_BLOCKED, 1); break; }
                             need = l + 1;
                         }
-                        if (G + need > admit_limit) { CADD(C_GATE_BLOCKED, 1); break; }
+                        if (G + need > admit_limit) {
+                            CADD(C_GATE_BLOCKED, 1);
+                            gate_closed = (a == 0) && (policy <= 1 || policy == 3);
+                            break;
+                        }
                         if (kExt && policy == 5) {
                             // MC benchmark (Section 4.1): start the queue head only if the usage of every future
                             // slot stays within M.  With a_i = l_i - (activation slot) + 1, request i holds a_i + tau
@@ -719,6 +730,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 // ---- overflow: evict the most recently activated until the slot fits (LIFO, Section 3.3);
                 //      evicted requests lose all progress and are again the head of the queue
                 if (G > M) {
+                    gate_closed = false;
                     CADD(C_OVERFLOW_STEPS, 1);
                     int nev = 0, wasted = 0;
                     if (policy == 3) {
@@ -861,6 +873,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     }
                     next_fin = __reduce_min_sync(FULL, cmin);
                     if (ndone > 0) {
+                        gate_closed = false;
                         nD += ndone;
                         Ndec -= ndone;
                         completed += ndone;
