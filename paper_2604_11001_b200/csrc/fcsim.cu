@@ -500,6 +500,8 @@ extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int per = max_steps_per_launch(h);
     const size_t smem_block = h->smem_block;
+    // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
+    CUDA_TRY(h, cudaFuncSetAttribute(h->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block));
     int left = n_steps;
     while (left > 0) {
         const int now = std::min(left, per);

@@ -191,3 +191,23 @@ def test_random_medium_configs(seed):
     cut = 1 + (seed * 97) % (cfg.T_max - 1)
     ref = orc.run(cfg, threads=4)
     assert_same(cfg, run_gpu(cfg, pieces=[cut, cfg.T_max - cut]), ref, cfg.T_max, cfg.name)
+
+
+def test_handles_with_different_shared_memory_needs_coexist():
+    # a handle that needs more than the default 48 KB of shared memory per CTA must keep working after a
+    # smaller one has been created (the opt-in limit belongs to the kernel, not to the handle)
+    from paper_2604_11001_b200 import binding as fb
+    big_cfg = degenerate_config(n=20, l=1, o=3, policy="greedy", b=0, K=0, c=0, M=100000, T=60, Qcap=2000, Acap=1500)
+    big_cfg = big_cfg.with_(decode=(wl.uniform_table(1, 40),))
+    small_cfg = wl.config1(replicas=4, T=60)
+    big = fb.Simulation(big_cfg)
+    assert big.launch_info()["smem_per_block"] > 48 * 1024
+    small = fb.Simulation(small_cfg)
+    small.run(60)
+    big.run(60)
+    small_c, _ = small.stats()
+    big_c, _ = big.stats()
+    assert (big_c == orc.run(big_cfg)["counters"]).all()
+    assert (small_c == orc.run(small_cfg)["counters"]).all()
+    big.close()
+    small.close()
