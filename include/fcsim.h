@@ -18,7 +18,9 @@
  * Conventions: every function returns 0 (FCSIM_OK) or a negative error code; nothing throws, aborts
  * or traps.  "HOST" / "DEVICE" says where a pointer must live.  Device output buffers are allocated
  * and owned by the caller; the library only allocates small private device copies of the tables.
- * One GPU; a handle is bound to the device that is current in fcsim_create.
+ * One GPU; a handle is bound to the device that is current in fcsim_create, and fcsim_run / fcsim_stats
+ * return FCSIM_EINVAL when called with another device current.  A handle is not thread-safe: calls on the
+ * same handle must not overlap.
  */
 #ifndef FCSIM_H
 #define FCSIM_H

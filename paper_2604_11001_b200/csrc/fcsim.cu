@@ -276,6 +276,14 @@ struct fcsim {
         }                                                 \
     } while (0)
 
+// A handle works on the device that was current in fcsim_create; calls made with another device current
+// are refused rather than silently launched on the wrong GPU.
+static int check_device(fcsim* h) {
+    int dev = -1;
+    CUDA_TRY(h, cudaGetDevice(&dev));
+    return dev == h->device ? FCSIM_OK : FCSIM_EINVAL;
+}
+
 extern "C" int fcsim_query_sizes(const fcsim_config* cfg, fcsim_sizes* out) {
     if (!out) return FCSIM_EINVAL;
     Layout L;
@@ -391,11 +399,16 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
 
     fcsim* h = new (std::nothrow) fcsim();
     if (!h) return FCSIM_ENOMEM;
+    try {
+        h->groups.assign(cfg->groups, cfg->groups + cfg->n_groups);
+    } catch (...) {
+        delete h;
+        return FCSIM_ENOMEM;
+    }
     h->cfg = *cfg;
     h->cfg.prompt = h->cfg.decode = nullptr;
     h->cfg.arrivals = nullptr;
     h->cfg.class_law.cdf = nullptr;
-    h->groups.assign(cfg->groups, cfg->groups + cfg->n_groups);
     h->cfg.groups = nullptr;
     h->L = L;
     h->buf = *b;
@@ -412,7 +425,11 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     e = cudaGetDeviceProperties(&prop, h->device);
     if (e != cudaSuccess) return fail(FCSIM_ECUDA);
     h->sm_count = prop.multiProcessorCount;
-    rc = upload_tables(h, cfg);
+    try {
+        rc = upload_tables(h, cfg);
+    } catch (...) {
+        rc = FCSIM_ENOMEM;
+    }
     if (rc != FCSIM_OK) return fail(rc);
 
     size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
@@ -497,6 +514,7 @@ static int max_steps_per_launch(const fcsim* h) {
 extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
     if (!h || n_steps < 0) return FCSIM_EINVAL;
     if ((long long)h->t_done + n_steps > h->cfg.T_max) return FCSIM_ERANGE;
+    if (int rc = check_device(h)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int per = max_steps_per_launch(h);
     const size_t smem_block = h->smem_block;
@@ -532,6 +550,7 @@ static double percentile(const long long* hist, int bins, int shift, long long n
 
 extern "C" int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_out, fcsim_summary* per_group_out) {
     if (!h) return FCSIM_EINVAL;
+    if (int rc = check_device(h)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int G = (int)h->groups.size();
     const int bins = h->cfg.hist_bins;
@@ -555,7 +574,11 @@ extern "C" int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_o
             launch_reduce_hist(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins, blocks, d_hist, st);
             CUDA_TRY(h, cudaGetLastError());
         }
-        host_scratch.resize(bytes / 8);
+        try {
+            host_scratch.resize(bytes / 8);
+        } catch (...) {
+            return FCSIM_ENOMEM;
+        }
         CUDA_TRY(h, cudaMemcpyAsync(host_scratch.data(), h->buf.scratch, bytes, cudaMemcpyDeviceToHost, st));
     }
     if (host_out)
