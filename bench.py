@@ -13,6 +13,7 @@ barrier when several ranks run).  One JSON line is printed by rank 0.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -117,8 +118,7 @@ def oracle_sample(workload: int, slots: int, n_rep: int):
     else:
         cfg = wl.PRESETS[workload]()
         per = max(1, n_rep // len(cfg.groups))
-        groups = tuple(wl.Group(g.policy, g.b_fp, g.chunk, g.arrivals_id, g.rng_replica_base,
-                                min(g.n_replicas, per)) for g in cfg.groups)
+        groups = tuple(dataclasses.replace(g, n_replicas=min(g.n_replicas, per)) for g in cfg.groups)
         sub = cfg.with_(groups=groups, T_max=slots)
     n = sub.n_replicas
     orc.lib()
