@@ -8,7 +8,6 @@ from __future__ import annotations
 
 import ctypes as C
 import os
-from dataclasses import dataclass
 from typing import List, Optional
 
 import numpy as np

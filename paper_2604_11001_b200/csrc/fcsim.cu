@@ -414,9 +414,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     h->buf = *b;
 
     auto fail = [&](int code) {
-        const int keep = h->last_cuda;
         release(h);
-        (void)keep;
         return code;
     };
     cudaError_t e = cudaGetDevice(&h->device);
