@@ -145,3 +145,10 @@ def test_one_call_split_into_several_launches():
     assert sim.launch_info()["max_steps_per_launch"] < 10000
     sim.close()
     _run_full(cfg, 10000, list(range(5, cfg.n_replicas, 16411)))
+
+
+def test_horizon_at_the_24_bit_limit():
+    # T_max = 2^24 - 1 slots: arrival times use all 24 bits of the packed entry, and the run spans 512 launches of
+    # 32 768 slots whose 32-bit partial sums are folded into the int64 counters
+    cfg = wl.config1(replicas=2, T=(1 << 24) - 1).with_(trace_stride=4096, complog_cap=4096, hist_shift=3)
+    _run_full(cfg, (1 << 24) - 1, [0, 1])
