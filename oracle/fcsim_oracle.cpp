@@ -3,7 +3,8 @@
 // Plain, slow, single-threaded CPU simulator of the token-level serving model of
 // Section 2.1 driven by the flow-controlled policy of Algorithm 2 (and by the greedy
 // prefill-first and chunked-prefill baselines named in the Introduction, and the alpha-protection
-// greedy baseline described in Section 4.1).  It is
+// greedy baseline described in Section 4.1; optionally with a preemption that keeps the generated
+// tokens, a variant the paper does not have).  It is
 // written directly from the paper, one request object at a time, with a std::deque
 // waiting queue and a std::vector active set; the KV usage U_t is re-summed from the
 // request objects every slot.  It shares no code, header or table with the CUDA
@@ -54,6 +55,10 @@ struct orc_group {
     const int32_t* b_class;  // CLASSFLOW (policy 4, Algorithm 1): activation budget b_k of every class
     int32_t mc_worst_case;   // MC: 0 = output lengths known, 1 = every request is projected with the longest
                              //     output length of its class (the unknown-length adaptation of Section 4.1)
+    int32_t preempt_keep;    // what an evicted request loses.  0 = everything (the model of Sections 2.1 and 3.3:
+                             //     the request is "refreshed").  1 = only its place in the cache: the j tokens it
+                             //     has generated are kept and become part of its prompt, (l, o) <- (l + j, o - j);
+                             //     this variant is not in the paper (recompute-style preemption of serving engines)
 };
 struct orc_config {
     int32_t M, K, T_max, Qcap, Acap;
@@ -190,6 +195,8 @@ int validate(const orc_config& c) {
         const orc_group& G = c.groups[g];
         if (G.policy < 0 || G.policy > 5 || G.n_replicas < 1) return -1;
         if (G.policy == 5 && (G.mc_worst_case < 0 || G.mc_worst_case > 1)) return -1;
+        if (G.preempt_keep < 0 || G.preempt_keep > 1) return -1;
+        if (G.preempt_keep && G.policy == 5) return -1;  // the MC benchmark never overflows: nothing to keep
         if (G.policy == 4) {
             if (!G.b_class) return -1;
             for (int k = 0; k < c.n_classes; ++k)
@@ -360,8 +367,19 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
                 Request r = P.back();
                 P.pop_back();
                 G -= (int64_t)r.p + r.j + (r.p == r.l ? 1 : 0);
-                C[C_WASTED_TOKENS] += r.j;
                 C[C_EVICTIONS]++;
+                if (grp.preempt_keep) {
+                    // The generated tokens stay with the request as prompt.  They are final, so they count as
+                    // delivered now, together with the workload they took: l*j + j(j+1)/2 = sum_{i<=j} (l + i),
+                    // which makes the workload of a request the sum over its segments,
+                    // w(l, o) = w(l, j) + w(l + j, o - j).
+                    C[C_COMPLETED_TOKENS] += r.j;
+                    C[C_SUM_W_COMPLETED] += (int64_t)r.l * r.j + (int64_t)r.j * (r.j + 1) / 2;
+                    r.l += r.j;
+                    r.o -= r.j;
+                } else {
+                    C[C_WASTED_TOKENS] += r.j;
+                }
                 r.p = 0;
                 r.j = 0;
                 Q.push_front(r);

@@ -167,6 +167,8 @@ class Group:
     m_admit: int = 0           # ALPHA: admission keeps usage <= m_admit = floor((1 - alpha) M)
     b_class: Tuple[int, ...] = ()  # CLASSFLOW: integer budget b_k of every class (Algorithm 1)
     mc_worst_case: int = 0         # MC: 1 = project every request with its class's longest output length
+    preempt_keep: int = 0          # 0 = an evicted request loses all progress (the paper's model); 1 = it keeps
+                                   # its generated tokens as prompt, (l, o) <- (l + j, o - j) (not in the paper)
 
 
 @dataclass(frozen=True)
@@ -376,12 +378,14 @@ def random_small_config(seed: int, n_replicas: int = 4, T: int = 60) -> SimConfi
                                      (int(rng.integers(0, 2 ** 31)), int(rng.integers(0, 2 ** 31)))))
     groups = []
     base = 0
+    keep_rng = np.random.default_rng(500_000 + seed)  # its own stream: the other parameters of a seed stay put
     for pol in (POLICY_FLOW, POLICY_GREEDY, POLICY_CHUNKED, POLICY_ALPHA, POLICY_CLASSFLOW, POLICY_MC):
         groups.append(Group(pol, b_fp=int(rng.integers(0, 3 * 65536)), chunk=int(rng.integers(1, 9)),
                             arrivals_id=int(rng.integers(0, 2)), rng_replica_base=base,
                             n_replicas=n_replicas, m_admit=int(rng.integers(max(2, M // 2), M + 1)),
                             b_class=tuple(int(x) for x in rng.integers(0, 3, size=n_classes)),
-                            mc_worst_case=int(rng.integers(0, 2))))
+                            mc_worst_case=int(rng.integers(0, 2)),
+                            preempt_keep=int(keep_rng.integers(0, 2)) if pol != POLICY_MC else 0))
         base += int(rng.integers(0, 2)) * n_replicas
     stride = int(rng.choice([1, 1, 2, 3]))
     return SimConfig(
@@ -402,12 +406,14 @@ def random_medium_config(seed: int, n_replicas: int = 2) -> SimConfig:
     omax = max(t.vmax for t in base.decode)
     M = int(rng.integers(lmax + omax, 6 * (lmax + omax)))
     groups = []
+    keep_rng = np.random.default_rng(600_000 + seed)
     for pol in rng.permutation(6)[:3]:
         groups.append(Group(int(pol), b_fp=int(rng.integers(0, 4 * 65536)), chunk=int(rng.choice([64, 512, 3000])),
                             arrivals_id=0, rng_replica_base=int(rng.integers(0, 1000)), n_replicas=n_replicas,
                             m_admit=int(rng.integers(M // 2, M + 1)),
                             b_class=tuple(int(x) for x in rng.integers(0, 3, size=base.n_classes)),
-                            mc_worst_case=int(rng.integers(0, 2))))
+                            mc_worst_case=int(rng.integers(0, 2)),
+                            preempt_keep=int(keep_rng.integers(0, 2)) if int(pol) != POLICY_MC else 0))
     lam = float(rng.uniform(0.2, 4.0))
     if rng.random() < 0.6:
         arr = Arrivals((poisson_table(lam),))

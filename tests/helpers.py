@@ -11,14 +11,14 @@ POLICIES = {"flow": wl.POLICY_FLOW, "greedy": wl.POLICY_GREEDY, "chunked": wl.PO
             "alpha": wl.POLICY_ALPHA, "mc": wl.POLICY_MC}
 
 
-def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, ma=0, **extra):
+def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, ma=0, keep=0, **extra):
     """Constant arrival count n per slot, constant lengths (l, o)."""
     pol = POLICIES[policy] if isinstance(policy, str) else policy
     return wl.SimConfig(
         M=M, K=K, T_max=T, Qcap=Qcap, Acap=Acap, seed=extra.pop("seed", 7),
         class_law=wl.constant_table(0), prompt=(wl.constant_table(l),), decode=(wl.constant_table(o),),
         arrivals=(wl.Arrivals((wl.constant_table(n),)),),
-        groups=(wl.Group(pol, b_fp=wl.b_to_fp(b), chunk=c, n_replicas=replicas, m_admit=ma),),
+        groups=(wl.Group(pol, b_fp=wl.b_to_fp(b), chunk=c, n_replicas=replicas, m_admit=ma, preempt_keep=keep),),
         trace_stride=1, hist_bins=extra.pop("hist_bins", 16), hist_shift=0, complog_cap=4 * T, **extra)
 
 

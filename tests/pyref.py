@@ -43,6 +43,7 @@ def brute_force(cfg, replica, n_steps):
         first += g.n_replicas
     key = (cfg.seed & M32, (cfg.seed >> 32) & M32)
     arr = cfg.arrivals[grp.arrivals_id]
+    keep = bool(getattr(grp, "preempt_keep", 0))
     reqs = []           # dicts: id, l, o, t_arr, status in {'wait','active','done'}, act_seq, p, j
     act_seq = 0
     state = 0
@@ -81,7 +82,7 @@ def brute_force(cfg, replica, n_steps):
                 if grp.policy == 5 and grp.mc_worst_case:
                     o_proj = cfg.decode[cls].vmin + len(cfg.decode[cls].cdf) - 1
                 reqs.append(dict(id=len(reqs), cls=cls, l=l, o=o, o_proj=o_proj, t_arr=t, status="wait",
-                                 act_seq=None, p=0, j=0))
+                                 act_seq=None, p=0, j=0, l0=l, o0=o, kept=0))
         n_dec_start = sum(1 for r in active() if r["p"] == r["l"])
         room = None if cfg.K == 0 else (max(0, cfg.K - n_dec_start) if grp.policy == 2 else cfg.K)
         if grp.policy == 2:
@@ -176,8 +177,13 @@ def brute_force(cfg, replica, n_steps):
             cnt["overflow_steps"] += 1
             while (active() if grp.policy == 3 else prospective() > cfg.M):   # alpha-protection evicts all
                 r = active()[-1]
-                cnt["wasted_tokens"] += r["j"]
                 cnt["evictions"] += 1
+                if keep:
+                    # the generated tokens stay with the request: it comes back with them in its prompt
+                    r["kept"] += r["j"]
+                    r["l"], r["o"] = r["l0"] + r["kept"], r["o0"] - r["kept"]
+                else:
+                    cnt["wasted_tokens"] += r["j"]
                 r["status"], r["p"], r["j"], r["act_seq"] = "wait", 0, 0, None
         for r in active():
             if r["p"] == r["l"]:
@@ -196,11 +202,19 @@ def brute_force(cfg, replica, n_steps):
                 cnt["completed"] += 1
                 cnt["sum_lat"] += lat
                 cnt["max_lat"] = max(cnt["max_lat"], lat)
-                cnt["completed_tokens"] += r["o"]
-                cnt["sum_w_completed"] += sum(r["l"] + jj for jj in range(1, r["o"] + 1))
+                if not keep:
+                    cnt["completed_tokens"] += r["o"]
+                    cnt["sum_w_completed"] += sum(r["l"] + jj for jj in range(1, r["o"] + 1))
         U_tr.append(U)
         Q_tr.append(len(waiting()))
         cnt["max_Q"] = max(cnt["max_Q"], len(waiting()))
+    if keep:
+        # tokens that can no longer be lost, request by request, in terms of the ORIGINAL lengths: all o0 of a
+        # finished request, the kept ones of the others; and the cache-slots those tokens occupied when made
+        for r in reqs:
+            n_final = r["o0"] if r["status"] == "done" else r["kept"]
+            cnt["completed_tokens"] += n_final
+            cnt["sum_w_completed"] += sum(r["l0"] + i for i in range(1, n_final + 1))
     cnt["q_final"] = len(waiting())
     cnt["p_final"] = len(active())
     cnt["resid_age"] = sum(n_steps - r["t_arr"] + 1 for r in reqs if r["status"] in ("wait", "active"))

@@ -25,9 +25,16 @@ def test_brute_force_agreement(seed):
 
 def test_random_configs_cover_every_branch():
     tot = np.zeros(orc.N_COUNTERS, dtype=np.int64)
+    keep_ev = np.zeros(6, dtype=np.int64)   # evictions under the keep-the-tokens variant, per policy
     for seed in range(30):
         cfg = wl.random_small_config(1000 + seed, n_replicas=2, T=50)
-        tot += orc.run(cfg)["counters"].sum(axis=0)
+        c = orc.run(cfg)["counters"]
+        tot += c.sum(axis=0)
+        for g, grp in enumerate(cfg.groups):
+            if grp.preempt_keep:
+                keep_ev[grp.policy] += c[2 * g:2 * g + 2, I["evictions"]].sum()
+                assert c[2 * g:2 * g + 2, I["wasted_tokens"]].sum() == 0
+    assert (keep_ev[:5] > 0).all(), keep_ev
     for name in ("dropped", "evictions", "gate_blocked_steps", "budget_blocked_steps", "acap_blocked_steps",
                  "wasted_tokens", "completed", "mmpp_state"):
         assert tot[I[name]] > 0, name
