@@ -88,7 +88,15 @@ typedef struct {
  * m_admit: ALPHA only, the admission limit floor((1 - alpha) M) in tokens, 1 .. M.
  * b_class: CLASSFLOW only, HOST array [n_classes] of the integer budgets b_k (0 .. 65535), borrowed during
  *       fcsim_create / fcsim_query_sizes; NULL otherwise.
- * mc_worst_case: MC only, 0 = output lengths known, 1 = project with the class's longest output length. */
+ * mc_worst_case: MC only, 0 = output lengths known, 1 = project with the class's longest output length.
+ * preempt_keep: what an evicted request loses.  0 = all progress: it re-enters the queue "refreshed", with
+ *       its original (l, o) and nothing generated (Sections 2.1 and 3.3; the paper's model).  1 = only its place
+ *       in the cache: the j output tokens it has generated stay with it as prompt, (l, o) <- (l + j, o - j), so
+ *       they are loaded again at its next activation instead of being generated again.  The paper has no such
+ *       variant.  The kept tokens are final, so completed_tokens grows by j and sum_w_completed by
+ *       l*j + j(j+1)/2 at the eviction (a request's workload is the sum over its segments), wasted_tokens
+ *       stays 0, and a completion record describes the last segment only.  Needs l_max + o_max <= 65536;
+ *       not accepted with MC, which never evicts (FCSIM_EINVAL). */
 typedef struct {
     int32_t policy;
     uint32_t b_fp;
@@ -99,6 +107,7 @@ typedef struct {
     int32_t m_admit;
     const int32_t* b_class;
     int32_t mc_worst_case;
+    int32_t preempt_keep;
 } fcsim_group;
 
 /* M: KV capacity in tokens (1 .. 2^30).  K: prefill-token budget per slot, 0 = none (the paper's model).

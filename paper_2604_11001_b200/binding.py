@@ -37,7 +37,8 @@ class fcsim_arrivals(C.Structure):
 class fcsim_group(C.Structure):
     _fields_ = [("policy", C.c_int32), ("b_fp", C.c_uint32), ("chunk", C.c_int32),
                 ("arrivals_id", C.c_int32), ("rng_replica_base", C.c_uint32), ("n_replicas", C.c_int32),
-                ("m_admit", C.c_int32), ("b_class", C.POINTER(C.c_int32)), ("mc_worst_case", C.c_int32)]
+                ("m_admit", C.c_int32), ("b_class", C.POINTER(C.c_int32)), ("mc_worst_case", C.c_int32),
+                ("preempt_keep", C.c_int32)]
 
 
 class fcsim_config(C.Structure):
@@ -162,7 +163,8 @@ def marshal_config(cfg):
             bptr = arr.ctypes.data_as(C.POINTER(C.c_int32))
         groups[i] = fcsim_group(int(g.policy), int(g.b_fp), int(g.chunk), int(g.arrivals_id),
                                 int(g.rng_replica_base), int(g.n_replicas), int(getattr(g, "m_admit", 0)), bptr,
-                                int(getattr(g, "mc_worst_case", 0)))
+                                int(getattr(g, "mc_worst_case", 0)),
+                                int(getattr(g, "preempt_keep", 0)))
     c = fcsim_config(int(cfg.M), int(cfg.K), int(cfg.T_max), int(cfg.Qcap), int(cfg.Acap), int(cfg.seed),
                      len(cfg.prompt), _mk_table(cfg.class_law, keep), prompt, decode, len(cfg.arrivals), arrs,
                      len(cfg.groups), groups, int(cfg.trace_stride), int(cfg.hist_bins), int(cfg.hist_shift),

@@ -87,6 +87,9 @@ int plan(const fcsim_config* c, Layout* L) {
         if (G.policy == FCSIM_POLICY_ALPHA && (G.m_admit < 1 || G.m_admit > c->M)) return FCSIM_EINVAL;
         if (G.arrivals_id < 0 || G.arrivals_id >= c->n_arrivals) return FCSIM_EINVAL;
         if (G.policy == FCSIM_POLICY_CHUNKED && G.chunk < 1) return FCSIM_EINVAL;
+        if (G.preempt_keep < 0 || G.preempt_keep > 1) return FCSIM_EINVAL;
+        // kept tokens join the prompt: l + j <= l_max + o_max - 1 must fit the entry's 16-bit prompt field
+        if (G.preempt_keep && (G.policy == FCSIM_POLICY_MC || lmax + omax > 65536)) return FCSIM_EINVAL;
         R += G.n_replicas;
     }
     if (R > 0x7fffffffLL) return FCSIM_EINVAL;
@@ -346,7 +349,7 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         }
         grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas,
                            G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M, boff,
-                           G.policy == FCSIM_POLICY_MC ? G.mc_worst_case : 0};
+                           G.policy == FCSIM_POLICY_MC ? G.mc_worst_case : 0, G.preempt_keep};
         first += G.n_replicas;
     }
     CUDA_TRY(h, cudaMalloc(&h->d_bclass, bclass.size() * sizeof(int32_t)));

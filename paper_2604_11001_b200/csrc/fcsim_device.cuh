@@ -67,6 +67,7 @@ struct DevGroup {
     int32_t admit_limit;  // usage a new admission may reach: M, or (1-alpha) M for the alpha-protection policy
     int32_t bclass_off;   // Algorithm 1: index of the group's per-class budgets in Params::bclass
     int32_t mc_worst;     // MC benchmark: project with the class's longest output length
+    int32_t keep;         // 1 = an evicted request keeps its generated tokens as prompt: (l, o) <- (l + j, o - j)
 };
 
 struct Params {
@@ -728,7 +729,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
 
                 // ---- overflow: evict the most recently activated until the slot fits (LIFO, Section 3.3);
-                //      evicted requests lose all progress and are again the head of the queue
+                //      evicted requests lose all progress (or, in the variant that keeps the generated tokens,
+                //      only their place in the cache) and are again the head of the queue
                 if (G > M) {
                     gate_closed = false;
                     CADD(C_OVERFLOW_STEPS, 1);
@@ -737,14 +739,29 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         // alpha-protection greedy (Section 4.1): every active request goes back to the queue.
                         // Completed entries were squeezed out above, so the whole active range is live and
                         // simply becomes the front of the queue.
+                        long long kept_w = 0;
                         for (int base = 0; base < nP; base += 32) {
                             const int i = base + lane;
                             if (i < nP) {
                                 const uint32_t sw = STATE(WA(shead + i));
-                                if (!(sw & kPrefillBit)) wasted += t - (int)sw + entry_o(RING(WR(head + i))) - 1;
+                                if (!(sw & kPrefillBit)) {
+                                    const uint64_t e = RING(WR(head + i));
+                                    const int j = t - (int)sw + entry_o(e) - 1;
+                                    wasted += j;
+                                    if (grp.keep != 0 && j > 0) {  // each lane rewrites its own entries only
+                                        const int l = entry_l(e);
+                                        kept_w += (long long)l * j + (long long)j * (j + 1) / 2;
+                                        RING(WR(head + i)) = pack_entry(l + j, entry_o(e) - j, entry_tarr(e), entry_cls(e));
+                                    }
+                                }
                             }
                         }
                         wasted = __reduce_add_sync(FULL, wasted);
+                        if (grp.keep != 0) {  // kept tokens are final: delivered now, with the workload they took
+                            CADD(C_COMPLETED_TOKENS, wasted);
+                            CADD(C_SUM_W_COMPLETED, warp_sum64(kept_w));
+                            wasted = 0;
+                        }
                         nev = nP;
                         nQ += nP;
                         nP = 0;
@@ -779,15 +796,26 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             }
                             __syncwarp();
                         }
-                        const uint64_t e = RING(WR(head + nP - 1));
+                        uint64_t e = RING(WR(head + nP - 1));
                         if (sw & kPrefillBit) {
                             G -= (int)(sw & ~kPrefillBit);
                             n_pref--;
                         } else {
                             const int j = t - (int)sw + entry_o(e) - 1;  // tokens generated before this slot
-                            G -= entry_l(e) + j + 1;
-                            wasted += j;
+                            const int l = entry_l(e);
+                            G -= l + j + 1;
                             Ndec--;
+                            if (grp.keep == 0) {
+                                wasted += j;
+                            } else if (j > 0) {
+                                // the generated tokens stay with the request as prompt; they are final, so they
+                                // are delivered now, with the workload they took: sum_{i<=j} (l + i)
+                                CADD(C_COMPLETED_TOKENS, j);
+                                CADD(C_SUM_W_COMPLETED, (long long)l * j + (long long)j * (j + 1) / 2);
+                                e = pack_entry(l + j, entry_o(e) - j, entry_tarr(e), entry_cls(e));
+                                __syncwarp();  // every lane has read the old entry
+                                if (lane == 0) RING(WR(head + nP - 1)) = e;
+                            }
                         }
                         q_e = e;
                         if ((kExt && policy == 4) && lane == 0) qcnt[entry_cls(e)] += 1;

@@ -211,3 +211,44 @@ def test_handles_with_different_shared_memory_needs_coexist():
     assert (small_c == orc.run(small_cfg)["counters"]).all()
     big.close()
     small.close()
+
+
+def test_evictions_that_keep_the_generated_tokens():
+    # every evicting policy on the heavy-tailed lengths of preset 5 and on preset 2's laws, many evictions,
+    # resumed launches (rewritten entries cross the save/restore of the rings), kept tokens next to 2^16
+    import dataclasses
+    base = wl.config5(replicas=1, T=6000)
+    groups = tuple(wl.Group(pol, b_fp=0x28000, chunk=256, n_replicas=3, m_admit=base.M - 64,
+                            b_class=(1, 1, 1), rng_replica_base=5, preempt_keep=1)
+                   for pol in (wl.POLICY_FLOW, wl.POLICY_GREEDY, wl.POLICY_CHUNKED, wl.POLICY_ALPHA,
+                               wl.POLICY_CLASSFLOW))
+    cfg = base.with_(groups=groups, trace_stride=1, complog_cap=4096)
+    ref = orc.run(cfg)
+    ev = ref["counters"][:, orc.CIDX["evictions"]].reshape(5, 3).sum(axis=1)
+    assert (ev > 50).all(), ev
+    assert ref["counters"][:, orc.CIDX["wasted_tokens"]].sum() == 0
+    assert_same(cfg, run_gpu(cfg, pieces=[1500, 7, 2493, 2000]), ref, 6000, "keep, preset-5 laws")
+    off = cfg.with_(groups=tuple(dataclasses.replace(g, preempt_keep=0) for g in groups))
+    assert (orc.run(off)["counters"] != ref["counters"]).any()
+    # longest lengths the variant accepts, l_max + o_max = 65536, with two running requests and a capacity that
+    # overflows 10 slots before the first one ends: the second is evicted holding 35 525 tokens, l becomes 65 525
+    big = degenerate_config(n=1, l=30000, o=35536, policy="greedy", b=0, K=0, c=0, M=131052, T=36000, Acap=2, keep=1)
+    big = big.with_(trace_stride=500, complog_cap=16)
+    refb = orc.run(big)
+    assert refb["counters"][0, orc.CIDX["evictions"]] == 1 and refb["counters"][0, orc.CIDX["completed"]] == 2
+    assert refb["counters"][0, orc.CIDX["completed_tokens"]] == 2 * 35536
+    assert refb["counters"][0, orc.CIDX["prefill_tokens"]] == 4 * 30000 + 65525
+    assert_same(big, run_gpu(big), refb, 36000, "keep, 16-bit edge")
+
+
+def test_keep_variant_argument_errors():
+    from paper_2604_11001_b200 import binding as fb
+    too_long = degenerate_config(n=1, l=30001, o=35536, policy="greedy", b=0, K=0, c=0, M=90000, T=10, keep=1)
+    with pytest.raises(fb.FcsimError):
+        fb.Simulation(too_long)
+    mc = degenerate_config(n=1, l=2, o=3, policy=wl.POLICY_MC, b=0, K=0, c=0, M=100, T=10, keep=1)
+    with pytest.raises(fb.FcsimError):
+        fb.Simulation(mc)
+    flag = degenerate_config(n=1, l=2, o=3, policy="greedy", b=0, K=0, c=0, M=100, T=10, keep=2)
+    with pytest.raises(fb.FcsimError):
+        fb.Simulation(flag)
