@@ -249,6 +249,8 @@ void launch_reduce_hist(const int* hist, const DevGroup* groups, int G, int R, i
 
 }  // namespace
 
+typedef void (*step_kernel_t)(const Params);
+
 struct fcsim {
     fcsim_config cfg;                 // scalar fields only; the pointers inside are not kept
     std::vector<fcsim_group> groups;  // host copy
@@ -259,7 +261,7 @@ struct fcsim {
     unsigned short* d_gpool = nullptr;
     int32_t* d_bclass = nullptr;
     size_t tabcache_off = 0, smem_block = 0;
-    void (*kernel)(const Params) = nullptr;  // step kernel variant for this configuration
+    step_kernel_t kernel = nullptr;  // step kernel variant for this configuration
     DevTable* d_tables = nullptr;
     DevArrivals* d_arrivals = nullptr;
     DevGroup* d_groups = nullptr;
@@ -433,34 +435,47 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     }
     if (rc != FCSIM_OK) return fail(rc);
 
-    size_t smem_block = (size_t)L.warps_per_block * L.smem_per_warp;
-    if (smem_block > (size_t)prop.sharedMemPerBlockOptin) return fail(FCSIM_ECAP);
-    {   // a copy of the table descriptors behind the warps' slices, if it does not cost a resident CTA
-        const size_t extra = align_up((size_t)(1 + 2 * cfg->n_classes) * sizeof(DevTable), 16);
-        const size_t sm = (size_t)prop.sharedMemPerMultiprocessor;
-        auto ctas = [&](size_t b) { return sm / (align_up(b, 1024) + 1024); };
-        h->tabcache_off = 0;
-        if (cfg->n_classes <= 16 && smem_block + extra <= (size_t)prop.sharedMemPerBlockOptin &&
-            ctas(smem_block + extra) == ctas(smem_block)) {
-            h->tabcache_off = smem_block;
-            smem_block += extra;
+    // Launch shape: warps per CTA (1 .. 4) and register allocation (<= 96 registers, or <= 80 with a few spilled
+    // words) are chosen for the largest number of resident warps per SM, as the occupancy calculator reports it
+    // for this device; ties go to the allocation without spills, then to the larger CTA.  A warp's slice of
+    // shared memory is fixed by the configuration, so small slices end up register-bound (6 CTAs of 4 warps at
+    // 80 registers) and large ones shared-memory-bound, where smaller CTAs waste less of the SM's 228 KB.
+    const bool ext = L.qcnt_off || L.has_v;
+    const size_t tab_extra = align_up((size_t)(1 + 2 * cfg->n_classes) * sizeof(DevTable), 16);
+    const size_t sm_bytes = (size_t)prop.sharedMemPerMultiprocessor;
+    auto ctas_by_smem = [&](size_t b) { return sm_bytes / (align_up(b, 1024) + 1024); };
+    int best_warps = 0, best_w = 0, best_occ = 0;
+    size_t best_block = 0, best_tab = 0;
+    for (int w = L.warps_per_block; w >= 1; --w) {
+        size_t block = (size_t)w * L.smem_per_warp, tab = 0;
+        if (block > (size_t)prop.sharedMemPerBlockOptin) continue;
+        // a copy of the table descriptors behind the warps' slices, if it does not cost a resident CTA
+        if (cfg->n_classes <= 16 && block + tab_extra <= (size_t)prop.sharedMemPerBlockOptin &&
+            ctas_by_smem(block + tab_extra) == ctas_by_smem(block)) {
+            tab = block;
+            block += tab_extra;
+        }
+        for (int six = 0; six <= 1; ++six) {
+            step_kernel_t k = ext ? (six ? fcsim_step_kernel<true, 6> : fcsim_step_kernel<true, 5>)
+                                  : (six ? fcsim_step_kernel<false, 6> : fcsim_step_kernel<false, 5>);
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
+            if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+            int occ = 0;
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, w * 32, block);
+            if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+            if (occ * w > best_warps) {
+                best_warps = occ * w; best_w = w; best_occ = occ; best_block = block; best_tab = tab;
+                h->kernel = k;
+            }
         }
     }
-    h->smem_block = smem_block;
-    // six CTAs per SM need <= 80 registers per thread and their shared memory (plus 1 KB each that the
-    // system reserves) within the SM's 228 KB; otherwise the 5-CTA register allocation is the better one
-    const bool six = 6 * (smem_block + 1024) <= (size_t)prop.sharedMemPerMultiprocessor;
-    if (L.qcnt_off || L.has_v)
-        h->kernel = six ? fcsim_step_kernel<true, 6> : fcsim_step_kernel<true, 5>;
-    else
-        h->kernel = six ? fcsim_step_kernel<false, 6> : fcsim_step_kernel<false, 5>;
-    e = cudaFuncSetAttribute(h->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block);
-    if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
-    int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, h->kernel, L.warps_per_block * 32, smem_block);
-    if (e != cudaSuccess || occ < 1) { h->last_cuda = (int)e; return fail(e != cudaSuccess ? FCSIM_ECUDA : FCSIM_ECAP); }
+    if (best_warps < 1) return fail(FCSIM_ECAP);
+    h->L.warps_per_block = best_w;
+    h->tabcache_off = best_tab;
+    h->smem_block = best_block;
+    const int occ = best_occ;
     h->blocks_per_sm = occ;
-    const long long want = (L.R + L.warps_per_block - 1) / L.warps_per_block;
+    const long long want = (L.R + h->L.warps_per_block - 1) / h->L.warps_per_block;
     h->grid = (int)std::max<long long>(1, std::min<long long>((long long)h->sm_count * occ, want));
 
     // zeroed buffers are the state "before slot 1"

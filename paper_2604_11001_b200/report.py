@@ -2,11 +2,12 @@
 throughput and token throughput (the metrics of Section 2.2) for every policy group of preset 6, at the
 horizons T = 1000, 2000, .., 10000, from one resumable GPU run.
 
-    python -m paper_2604_11001_b200.report [--replicas 1024]
+    python -m paper_2604_11001_b200.report [--replicas 1024] [--rate 15] [--keep-tokens]
 """
 from __future__ import annotations
 
 import argparse
+import dataclasses
 
 from . import binding as fb
 from . import workloads as wl
@@ -15,8 +16,12 @@ NAMES = ("Algorithm 2, b=12", "greedy + LIFO eviction", "alpha-protection greedy
          "MC, known lengths", "MC, worst-case lengths")
 
 
-def run(replicas: int = 1024, horizons=range(1000, 10001, 1000), device: str = "cuda:0", total_rate: float = 5.0):
+def run(replicas: int = 1024, horizons=range(1000, 10001, 1000), device: str = "cuda:0", total_rate: float = 5.0,
+        keep_tokens: bool = False):
     cfg = wl.config6(replicas=replicas, T=max(horizons), total_rate=total_rate)
+    if keep_tokens:  # evicted requests keep their generated tokens as prompt (not the paper's rule); MC never evicts
+        cfg = cfg.with_(groups=tuple(g if g.policy == wl.POLICY_MC else dataclasses.replace(g, preempt_keep=1)
+                                     for g in cfg.groups))
     sim = fb.Simulation(cfg, device=device)
     rows = []
     for T in horizons:
@@ -34,8 +39,10 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--replicas", type=int, default=1024)
     ap.add_argument("--rate", type=float, default=5.0, help="total arrivals per slot (5 = total, 15 = 5 per class)")
+    ap.add_argument("--keep-tokens", action="store_true",
+                    help="evicted requests keep their generated tokens as prompt instead of being refreshed")
     args = ap.parse_args()
-    rows = run(args.replicas, total_rate=args.rate)
+    rows = run(args.replicas, total_rate=args.rate, keep_tokens=args.keep_tokens)
     print("%6s  %-26s %12s %12s %14s %14s %10s %10s" % ("T", "policy", "mean lat", "p95 lat", "requests/slot",
                                                           "tokens/slot", "evictions", "dropped"))
     for r in rows:
