@@ -353,6 +353,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         // memory is released (a completion or an eviction): the usage only grows and the head does not change.
         // While the flag is up a slot's activation attempt is just counted as refused.
         bool gate_closed = false;
+        bool mc_refused = false;  // MC benchmark: the last future-memory test refused the queue head
         // statistics of completions, private to the lane that saw them; reduced once when the replica is put back
         unsigned long long acc_lat = 0, acc_w = 0;
         uint32_t acc_o = 0, completed = 0;
@@ -671,8 +672,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                                       (int)tabs[1 + p.n_classes + entry_cls(eh)].n - 1)
                                                    : entry_o(eh);
                             const int f_h = t + op_h - 1, a_h = l - t + 1;
+                            // One pass tests the head and, tentatively, already books it on every earlier last
+                            // slot; a refusal takes the booking back in a second pass.  Right after a refusal
+                            // the next test is expected to fail too and runs read-only, booking only if it passes.
+                            const bool tentative = !mc_refused;
                             bool ok = true;
                             long long S = 0;
+#pragma unroll 2
                             for (int base = 0; base < nP; base += 32) {
                                 const int i = base + lane;
                                 const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
@@ -682,25 +688,35 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     if (worst) f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
                                                       (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
                                     const int a_i = entry_l(ei) + entry_o(ei) - (int)swi;
-                                    if (f_i <= f_h && (long long)vproj[WA(shead + i)] + a_h + f_i > M) ok = false;
+                                    if (f_i <= f_h) {
+                                        // <= M + 2 * 65536 < 2^31: no overflow
+                                        const int v = vproj[WA(shead + i)] + a_h + f_i;
+                                        if (v > M) ok = false;
+                                        if (tentative) vproj[WA(shead + i)] = v;
+                                    }
                                     if (f_i >= f_h) S += a_i + f_h;
                                 }
                             }
                             S = warp_sum64(S) + a_h + f_h;
-                            if (__any_sync(FULL, !ok) || S > M) { CADD(C_GATE_BLOCKED, 1); break; }
-                            for (int base = 0; base < nP; base += 32) {   // it starts: it adds to every earlier last slot
-                                const int i = base + lane;
-                                const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
-                                if (swi != kDead) {
-                                    int f_i = (int)swi;
-                                    if (worst) {
-                                        const uint64_t ei = RING(WR(head + i));
-                                        f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
-                                               (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
+                            const bool fits = !__any_sync(FULL, !ok) && S <= M;
+                            if (fits != tentative) {  // take the booking back, or make the one the read-only test skipped
+#pragma unroll 2
+                                for (int base = 0; base < nP; base += 32) {
+                                    const int i = base + lane;
+                                    const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
+                                    if (swi != kDead) {
+                                        int f_i = (int)swi;
+                                        if (worst) {
+                                            const uint64_t ei = RING(WR(head + i));
+                                            f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
+                                                   (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
+                                        }
+                                        if (f_i <= f_h) vproj[WA(shead + i)] += fits ? (a_h + f_i) : -(a_h + f_i);
                                     }
-                                    if (f_i <= f_h) vproj[WA(shead + i)] += a_h + f_i;
                                 }
                             }
+                            mc_refused = !fits;
+                            if (!fits) { CADD(C_GATE_BLOCKED, 1); break; }
                             if (lane == 0) vproj[WA(shead + nP)] = (int)S;
                         }
                         uint32_t sw;
@@ -840,6 +856,27 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 //      are taken now, their entries are only marked and squeezed out later in bulk
                 if ((uint32_t)t == next_fin) {
                     int ndone = 0, sum_lo = 0;
+                    int pend_f = 0, pend_a = 0, npend = 0;  // lane q < npend: projected last slot and offset of an early finisher
+                    auto mc_release = [&]() {
+                        __syncwarp();  // the finishers' state words are marked
+                        for (int vb = 0; vb < nP; vb += 32) {
+                            const int vi = vb + lane;
+                            const uint32_t swv = (vi < nP) ? STATE(WA(shead + vi)) : kDead;
+                            int f_v = 0x3fffffff;  // later than any slot: a completed entry takes no correction
+                            if (swv != kDead) {
+                                const uint64_t ev = RING(WR(head + vi));
+                                const DevTable dv = tabs[1 + p.n_classes + entry_cls(ev)];
+                                f_v = (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev);
+                            }
+                            int delta = 0;
+                            for (int q = 0; q < npend; ++q) {
+                                const int f_c = __shfl_sync(FULL, pend_f, q), a_c = __shfl_sync(FULL, pend_a, q);
+                                if (f_v <= f_c) delta += a_c + f_v;
+                            }
+                            if (delta != 0) vproj[WA(shead + vi)] -= delta;
+                        }
+                        npend = 0;
+                    };
                     uint32_t due = __ballot_sync(FULL, cmin == (uint32_t)t);
                     while (due) {
                         const int c = __ffs(due) - 1;
@@ -872,33 +909,28 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 ndone += __popc(m);
                                 if (kExt && policy == 5 && grp.mc_worst != 0) {
                                     // MC benchmark with worst-case projection: a request that ends before its
-                                    // projected last slot f_c leaves the projected usage of every last slot <= f_c
-                                    __syncwarp();
-                                    uint32_t fm = m;
-                                    while (fm) {
-                                        const int src = __ffs(fm) - 1;
-                                        fm &= fm - 1;
-                                        const uint64_t ec = __shfl_sync(FULL, e, src);
+                                    // projected last slot f_c leaves the projected usage of every last slot <= f_c.
+                                    // The slot's early finishers are collected, one per lane, and taken out of the
+                                    // projections in one pass over the active range.
+                                    const int cntm = __popc(m);
+                                    if (npend + cntm > 32) mc_release();
+                                    const int rnk = lane - npend;
+                                    const bool take = rnk >= 0 && rnk < cntm;
+                                    const int src = take ? (int)__fns(m, 0, rnk + 1) : 0;
+                                    const uint64_t ec = __shfl_sync(FULL, e, src);
+                                    if (take) {
                                         const DevTable dc = tabs[1 + p.n_classes + entry_cls(ec)];
-                                        const int f_c = t - entry_o(ec) + dc.vmin + (int)dc.n - 1;
-                                        const int a_c = entry_l(ec) + entry_o(ec) - t;
-                                        for (int vb = 0; vb < nP; vb += 32) {
-                                            const int vi = vb + lane;
-                                            const uint32_t swv = (vi < nP) ? STATE(WA(shead + vi)) : kDead;
-                                            if (swv != kDead) {
-                                                const uint64_t ev = RING(WR(head + vi));
-                                                const DevTable dv = tabs[1 + p.n_classes + entry_cls(ev)];
-                                                const int f_v = (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev);
-                                                if (f_v <= f_c) vproj[WA(shead + vi)] -= a_c + f_v;
-                                            }
-                                        }
+                                        pend_f = t - entry_o(ec) + dc.vmin + (int)dc.n - 1;
+                                        pend_a = entry_l(ec) + entry_o(ec) - t;
                                     }
+                                    npend += cntm;
                                 }
                             }
                             gmin = min(gmin, __reduce_min_sync(FULL, (done || sw == kDead) ? kNoFin : sw));
                         }
                         if (lane == c) cmin = gmin;
                     }
+                    if (kExt && npend > 0) mc_release();
                     next_fin = __reduce_min_sync(FULL, cmin);
                     if (ndone > 0) {
                         gate_closed = false;

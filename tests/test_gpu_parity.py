@@ -252,3 +252,18 @@ def test_keep_variant_argument_errors():
     flag = degenerate_config(n=1, l=2, o=3, policy="greedy", b=0, K=0, c=0, M=100, T=10, keep=2)
     with pytest.raises(fb.FcsimError):
         fb.Simulation(flag)
+
+
+def test_mc_many_finishers_in_one_slot():
+    # worst-case projection with more than 32 requests ending in the same slot (their corrections are collected
+    # one per lane and flushed when the lanes run out), with and without a binding capacity
+    for M, mode in ((100000, 1), (330, 1), (330, 0)):
+        cfg = degenerate_config(n=48, l=1, o=3, policy=wl.POLICY_MC, b=0, K=0, c=0, M=M, T=300, Qcap=600, Acap=400)
+        cfg = cfg.with_(decode=(wl.uniform_table(1, 4),), arrivals=(wl.Arrivals((wl.poisson_table(44.0),)),),
+                        groups=(wl.Group(wl.POLICY_MC, n_replicas=3, mc_worst_case=mode),), complog_cap=20000)
+        ref = orc.run(cfg)
+        c = ref["counters"]
+        assert (c[:, orc.CIDX["completed"]] > 32 * 150).all()
+        if M == 330:
+            assert (c[:, orc.CIDX["gate_blocked_steps"]] > 50).all()
+        assert_same(cfg, run_gpu(cfg, pieces=[100, 200]), ref, 300, f"MC finishers M={M} worst={mode}")
