@@ -32,9 +32,9 @@ UNIT = "replica-steps/s"
 # Executed warp-instructions per replica-step of the step kernel in the timed regime of each preset,
 # from the committed ncu captures (profiles/): smsp__inst_executed.sum / (replicas x slots) of one launch.
 # None = not captured for the current kernel.
-INST_PER_REPLICA_STEP = {1: 269.7, 2: 310.5, 3: 357.8, 4: 446.7, 5: 256.7, 6: 3025.0}
+INST_PER_REPLICA_STEP = {1: 270.8, 2: 311.7, 3: 357.5, 4: 446.9, 5: 258.4, 6: 2303.4}
 # DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
-DRAM_BYTES_PER_REPLICA_STEP = {1: 0.03, 2: 22.9, 3: 17.9, 4: 10.0, 5: 7.9, 6: 79.6}
+DRAM_BYTES_PER_REPLICA_STEP = {1: 29.1, 2: 22.9, 3: 17.8, 4: 10.0, 5: 7.9, 6: 79.6}
 
 DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000, 6: 500}
 NAMES = {1: "cfg1-tiny-flow", 2: "cfg2-policy-comparison", 3: "cfg3-stability-sweep", 4: "cfg4-heavy-tail",
