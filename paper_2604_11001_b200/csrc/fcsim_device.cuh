@@ -678,24 +678,30 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             const bool tentative = !mc_refused;
                             bool ok = true;
                             long long S = 0;
-#pragma unroll 2
+#pragma unroll 4
                             for (int base = 0; base < nP; base += 32) {
+                                // loads first and unconditionally (lanes past the range read entry 0 and ignore
+                                // it), so that the iterations' shared-memory round trips overlap
                                 const int i = base + lane;
-                                const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
-                                if (swi != kDead) {
-                                    const uint64_t ei = RING(WR(head + i));
-                                    int f_i = (int)swi;
-                                    if (worst) f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
-                                                      (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
-                                    const int a_i = entry_l(ei) + entry_o(ei) - (int)swi;
-                                    if (f_i <= f_h) {
-                                        // <= M + 2 * 65536 < 2^31: no overflow
-                                        const int v = vproj[WA(shead + i)] + a_h + f_i;
-                                        if (v > M) ok = false;
-                                        if (tentative) vproj[WA(shead + i)] = v;
-                                    }
-                                    if (f_i >= f_h) S += a_i + f_h;
+                                const bool in = i < nP;
+                                const int si = WA(shead + (in ? i : 0));
+                                const uint32_t swi = STATE(si);
+                                const uint64_t ei = RING(WR(head + (in ? i : 0)));
+                                const uint32_t vi = (uint32_t)vproj[si];
+                                const bool live = in && swi != kDead;
+                                uint32_t f_i = swi;
+                                if (worst) {
+                                    const DevTable d = tabs[1 + p.n_classes + (live ? entry_cls(ei) : 0)];
+                                    f_i += (uint32_t)(d.vmin + (int)d.n - 1 - entry_o(ei));
                                 }
+                                // unsigned arithmetic: ignored lanes may hold anything; for live entries
+                                // v <= M + 2 * 65536 < 2^31
+                                const int v = (int)(vi + (uint32_t)a_h + f_i);
+                                if (live && (int)f_i <= f_h) {
+                                    if (v > M) ok = false;
+                                    if (tentative) vproj[si] = v;
+                                }
+                                if (live && (int)f_i >= f_h) S += (int)((uint32_t)(entry_l(ei) + entry_o(ei)) - swi + (uint32_t)f_h);
                             }
                             S = warp_sum64(S) + a_h + f_h;
                             const bool fits = !__any_sync(FULL, !ok) && S <= M;
@@ -859,21 +865,23 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     int pend_f = 0, pend_a = 0, npend = 0;  // lane q < npend: projected last slot and offset of an early finisher
                     auto mc_release = [&]() {
                         __syncwarp();  // the finishers' state words are marked
+#pragma unroll 2
                         for (int vb = 0; vb < nP; vb += 32) {
                             const int vi = vb + lane;
-                            const uint32_t swv = (vi < nP) ? STATE(WA(shead + vi)) : kDead;
-                            int f_v = 0x3fffffff;  // later than any slot: a completed entry takes no correction
-                            if (swv != kDead) {
-                                const uint64_t ev = RING(WR(head + vi));
-                                const DevTable dv = tabs[1 + p.n_classes + entry_cls(ev)];
-                                f_v = (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev);
-                            }
+                            const bool in = vi < nP;
+                            const int si = WA(shead + (in ? vi : 0));
+                            const uint32_t swv = STATE(si);
+                            const uint64_t ev = RING(WR(head + (in ? vi : 0)));
+                            const bool live = in && swv != kDead;
+                            const DevTable dv = tabs[1 + p.n_classes + (live ? entry_cls(ev) : 0)];
+                            // a completed entry takes no correction: later than any slot
+                            const int f_v = live ? (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev) : 0x3fffffff;
                             int delta = 0;
                             for (int q = 0; q < npend; ++q) {
                                 const int f_c = __shfl_sync(FULL, pend_f, q), a_c = __shfl_sync(FULL, pend_a, q);
                                 if (f_v <= f_c) delta += a_c + f_v;
                             }
-                            if (delta != 0) vproj[WA(shead + vi)] -= delta;
+                            if (delta != 0) vproj[si] -= delta;
                         }
                         npend = 0;
                     };
