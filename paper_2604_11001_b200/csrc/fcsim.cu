@@ -251,6 +251,41 @@ void launch_reduce_hist(const int* hist, const DevGroup* groups, int G, int R, i
 
 typedef void (*step_kernel_t)(const Params);
 
+// The step kernel compiled for one policy, for a register allocation that lets 6 or 5 CTAs reside on an SM, and
+// for what is recorded per slot (0 nothing, 1 trace only, 2 decided at run time; Algorithm 1 and the MC benchmark
+// exist in the run-time form only).
+template <int kPol>
+static step_kernel_t step_kernel_for(bool six, int rec) {
+    if (kPol >= 4 || rec == 2) return six ? fcsim_step_kernel<kPol, 6, 2> : fcsim_step_kernel<kPol, 5, 2>;
+    constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 and 5 uninstantiated
+    if (rec == 1) return six ? fcsim_step_kernel<kP, 6, 1> : fcsim_step_kernel<kP, 5, 1>;
+    return six ? fcsim_step_kernel<kP, 6, 0> : fcsim_step_kernel<kP, 5, 0>;
+}
+static step_kernel_t pick_step_kernel(int policy, bool six, int rec) {
+    switch (policy) {
+        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(six, rec);
+        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(six, rec);
+        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(six, rec);
+        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(six, rec);
+        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(six, rec);
+        case FCSIM_POLICY_MC: return step_kernel_for<5>(six, rec);
+        default: return nullptr;
+    }
+}
+
+// One launch per policy present in the configuration: its kernel, its groups (a contiguous piece of the
+// policy-sorted group array), its launch shape, and the side stream it runs on when there are several.
+struct PolicyLaunch {
+    int policy = 0;
+    step_kernel_t kernel = nullptr;
+    int pg_off = 0, pg_cnt = 0;   // its groups in d_pgroups
+    int n_work = 0;               // replicas
+    int warps_per_block = 0, blocks_per_sm = 0, grid = 0;
+    size_t smem_block = 0, tabcache_off = 0;
+    cudaStream_t side = nullptr;  // null: the caller's stream
+    cudaEvent_t done = nullptr;
+};
+
 struct fcsim {
     fcsim_config cfg;                 // scalar fields only; the pointers inside are not kept
     std::vector<fcsim_group> groups;  // host copy
@@ -260,13 +295,15 @@ struct fcsim {
     uint32_t* d_pool = nullptr;
     unsigned short* d_gpool = nullptr;
     int32_t* d_bclass = nullptr;
-    size_t tabcache_off = 0, smem_block = 0;
-    step_kernel_t kernel = nullptr;  // step kernel variant for this configuration
+    std::vector<PolicyLaunch> launches;  // most expensive policy first
+    int main_launch = 0;                 // the launch with the most replicas (reported by fcsim_get_launch_info)
+    cudaEvent_t fork = nullptr;
+    DevGroup* d_pgroups = nullptr;       // the groups sorted by policy (stable), with their work-item offsets
     DevTable* d_tables = nullptr;
     DevArrivals* d_arrivals = nullptr;
     DevGroup* d_groups = nullptr;
     unsigned int* d_work = nullptr;
-    int device = 0, sm_count = 0, blocks_per_sm = 1, grid = 1;
+    int device = 0, sm_count = 0;
     int t_done = 0;
     int last_cuda = 0;
     size_t table_bytes = 0;
@@ -351,8 +388,24 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         }
         grps[g] = DevGroup{G.policy, G.b_fp, G.chunk, G.arrivals_id, G.rng_replica_base, first, G.n_replicas,
                            G.policy == FCSIM_POLICY_ALPHA ? G.m_admit : c->M, boff,
-                           G.policy == FCSIM_POLICY_MC ? G.mc_worst_case : 0, G.preempt_keep};
+                           G.policy == FCSIM_POLICY_MC ? G.mc_worst_case : 0, G.preempt_keep, first};
         first += G.n_replicas;
+    }
+    // the same groups sorted by policy (order within a policy kept): one launch per policy walks its piece
+    std::vector<DevGroup> pgrps;
+    for (int pol = FCSIM_POLICY_MC; pol >= FCSIM_POLICY_FLOW; --pol) {  // costly policies first
+        PolicyLaunch pl;
+        pl.policy = pol;
+        pl.pg_off = (int)pgrps.size();
+        for (int g = 0; g < c->n_groups; ++g) {
+            if (grps[g].policy != pol) continue;
+            DevGroup d = grps[g];
+            d.wfirst = pl.n_work;
+            pl.n_work += d.n;
+            pgrps.push_back(d);
+        }
+        pl.pg_cnt = (int)pgrps.size() - pl.pg_off;
+        if (pl.pg_cnt > 0) h->launches.push_back(pl);
     }
     CUDA_TRY(h, cudaMalloc(&h->d_bclass, bclass.size() * sizeof(int32_t)));
     CUDA_TRY(h, cudaMemcpy(h->d_bclass, bclass.data(), bclass.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
@@ -362,6 +415,8 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
     CUDA_TRY(h, cudaMalloc(&h->d_tables, tables.size() * sizeof(DevTable)));
     CUDA_TRY(h, cudaMalloc(&h->d_arrivals, arrs.size() * sizeof(DevArrivals)));
     CUDA_TRY(h, cudaMalloc(&h->d_groups, grps.size() * sizeof(DevGroup)));
+    CUDA_TRY(h, cudaMalloc(&h->d_pgroups, pgrps.size() * sizeof(DevGroup)));
+    CUDA_TRY(h, cudaMemcpy(h->d_pgroups, pgrps.data(), pgrps.size() * sizeof(DevGroup), cudaMemcpyHostToDevice));
     CUDA_TRY(h, cudaMalloc(&h->d_work, 16 * sizeof(unsigned int)));
     CUDA_TRY(h, cudaMemset(h->d_work, 0, 16 * sizeof(unsigned int)));
     CUDA_TRY(h, cudaMemcpy(h->d_pool, pool.data(), pool.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
@@ -381,6 +436,12 @@ static void release(fcsim* h) {
     cudaFree(h->d_tables);
     cudaFree(h->d_arrivals);
     cudaFree(h->d_groups);
+    cudaFree(h->d_pgroups);
+    for (PolicyLaunch& pl : h->launches) {
+        if (pl.done) cudaEventDestroy(pl.done);
+        if (pl.side) cudaStreamDestroy(pl.side);
+    }
+    if (h->fork) cudaEventDestroy(h->fork);
     cudaFree(h->d_work);
     delete h;
 }
@@ -435,48 +496,66 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     }
     if (rc != FCSIM_OK) return fail(rc);
 
-    // Launch shape: warps per CTA (1 .. 4) and register allocation (<= 96 registers, or <= 80 with a few spilled
-    // words) are chosen for the largest number of resident warps per SM, as the occupancy calculator reports it
-    // for this device; ties go to the allocation without spills, then to the larger CTA.  A warp's slice of
-    // shared memory is fixed by the configuration, so small slices end up register-bound (6 CTAs of 4 warps at
-    // 80 registers) and large ones shared-memory-bound, where smaller CTAs waste less of the SM's 228 KB.
+    // Launch shape, per policy kernel: warps per CTA (1 .. 4) and register allocation (<= 96 registers, or <= 80)
+    // are chosen for the largest number of resident warps per SM, as the occupancy calculator reports it for this
+    // device; ties go to the roomier register allocation, then to the larger CTA.  A warp's slice of shared memory
+    // is fixed by the configuration, so small slices end up register-bound (6 CTAs of 4 warps at 80 registers)
+    // and large ones shared-memory-bound, where smaller CTAs waste less of the SM's 228 KB.
     const bool ext = L.qcnt_off || L.has_v;
+    // what is recorded per slot is a compile-time property of the kernels of the common policies
+    const int rec = (ext || cfg->complog_cap > 0 || L.tstage_off != 0) ? 2 : (L.n_rec > 0 ? 1 : 0);
     const size_t tab_extra = align_up((size_t)(1 + 2 * cfg->n_classes) * sizeof(DevTable), 16);
     const size_t sm_bytes = (size_t)prop.sharedMemPerMultiprocessor;
     auto ctas_by_smem = [&](size_t b) { return sm_bytes / (align_up(b, 1024) + 1024); };
-    int best_warps = 0, best_w = 0, best_occ = 0;
-    size_t best_block = 0, best_tab = 0;
-    for (int w = L.warps_per_block; w >= 1; --w) {
-        size_t block = (size_t)w * L.smem_per_warp, tab = 0;
-        if (block > (size_t)prop.sharedMemPerBlockOptin) continue;
-        // a copy of the table descriptors behind the warps' slices, if it does not cost a resident CTA
-        if (cfg->n_classes <= 16 && block + tab_extra <= (size_t)prop.sharedMemPerBlockOptin &&
-            ctas_by_smem(block + tab_extra) == ctas_by_smem(block)) {
-            tab = block;
-            block += tab_extra;
-        }
-        for (int six = 0; six <= 1; ++six) {
-            step_kernel_t k = ext ? (six ? fcsim_step_kernel<true, 6> : fcsim_step_kernel<true, 5>)
-                                  : (six ? fcsim_step_kernel<false, 6> : fcsim_step_kernel<false, 5>);
-            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
-            if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
-            int occ = 0;
-            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, w * 32, block);
-            if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
-            if (occ * w > best_warps) {
-                best_warps = occ * w; best_w = w; best_occ = occ; best_block = block; best_tab = tab;
-                h->kernel = k;
+    size_t most_work = 0;
+    for (size_t li = 0; li < h->launches.size(); ++li) {
+        PolicyLaunch& pl = h->launches[li];
+        int best_warps = 0;
+        for (int w = L.warps_per_block; w >= 1; --w) {
+            size_t block = (size_t)w * L.smem_per_warp, tab = 0;
+            if (block > (size_t)prop.sharedMemPerBlockOptin) continue;
+            // a copy of the table descriptors behind the warps' slices, if it does not cost a resident CTA
+            if (cfg->n_classes <= 16 && block + tab_extra <= (size_t)prop.sharedMemPerBlockOptin &&
+                ctas_by_smem(block + tab_extra) == ctas_by_smem(block)) {
+                tab = block;
+                block += tab_extra;
+            }
+            for (int six = 0; six <= 1; ++six) {
+                step_kernel_t k = pick_step_kernel(pl.policy, six != 0, rec);
+                if (!k) return fail(FCSIM_EINVAL);
+                e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
+                if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+                int occ = 0;
+                e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, w * 32, block);
+                if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+                if (occ * w > best_warps) {
+                    best_warps = occ * w;
+                    pl.kernel = k;
+                    pl.warps_per_block = w;
+                    pl.blocks_per_sm = occ;
+                    pl.smem_block = block;
+                    pl.tabcache_off = tab;
+                }
             }
         }
+        if (best_warps < 1) return fail(FCSIM_ECAP);
+        const long long want = ((long long)pl.n_work + pl.warps_per_block - 1) / pl.warps_per_block;
+        pl.grid = (int)std::max<long long>(1, std::min<long long>((long long)h->sm_count * pl.blocks_per_sm, want));
+        if ((size_t)pl.n_work > most_work) { most_work = (size_t)pl.n_work; h->main_launch = (int)li; }
     }
-    if (best_warps < 1) return fail(FCSIM_ECAP);
-    h->L.warps_per_block = best_w;
-    h->tabcache_off = best_tab;
-    h->smem_block = best_block;
-    const int occ = best_occ;
-    h->blocks_per_sm = occ;
-    const long long want = (L.R + h->L.warps_per_block - 1) / h->L.warps_per_block;
-    h->grid = (int)std::max<long long>(1, std::min<long long>((long long)h->sm_count * occ, want));
+    // several policies: their launches run side by side (the first on the caller's stream, the others on streams
+    // of the handle, forked from and joined to the caller's stream by events), so that no SM idles while the last
+    // replicas of one policy finish
+    if (h->launches.size() > 1) {
+        e = cudaEventCreateWithFlags(&h->fork, cudaEventDisableTiming);
+        if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+        for (size_t li = 1; li < h->launches.size(); ++li) {
+            e = cudaStreamCreateWithFlags(&h->launches[li].side, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->launches[li].done, cudaEventDisableTiming);
+            if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+        }
+    }
+    h->L.warps_per_block = h->launches[h->main_launch].warps_per_block;
 
     // zeroed buffers are the state "before slot 1"
     const struct { void* p; size_t n; } z[] = {{b->workspace, sz.workspace}, {b->counters, sz.counters},
@@ -505,9 +584,9 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.qcnt_off = (uint32_t)L.qcnt_off;
     p.tstage_off = (uint32_t)L.tstage_off;
     p.state_bytes = (uint32_t)L.state_bytes;
-    p.tabcache_off = (uint32_t)h->tabcache_off;
     p.has_v = L.has_v;
-    p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals; p.groups = h->d_groups;
+    p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals;
+    p.groups = h->d_pgroups;  // narrowed to the policy's piece at every launch
     p.workspace = static_cast<unsigned char*>(b->workspace);
     p.ws_stride = L.ws_stride;
     p.counters = static_cast<long long*>(b->counters);
@@ -533,18 +612,30 @@ extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
     if (int rc = check_device(h)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int per = max_steps_per_launch(h);
-    const size_t smem_block = h->smem_block;
-    // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
-    CUDA_TRY(h, cudaFuncSetAttribute(h->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_block));
     int left = n_steps;
     while (left > 0) {
         const int now = std::min(left, per);
-        Params p = h->params;
-        p.t0 = h->t_done;
-        p.n_steps = now;
-        CUDA_TRY(h, cudaMemsetAsync(h->d_work, 0, sizeof(unsigned int), st));
-        h->kernel<<<h->grid, h->L.warps_per_block * 32, smem_block, st>>>(p);
-        CUDA_TRY(h, cudaGetLastError());
+        CUDA_TRY(h, cudaMemsetAsync(h->d_work, 0, 8 * sizeof(unsigned int), st));  // one work counter per policy
+        if (h->launches.size() > 1) CUDA_TRY(h, cudaEventRecord(h->fork, st));
+        for (const PolicyLaunch& pl : h->launches) {
+            cudaStream_t ls = pl.side ? pl.side : st;
+            if (pl.side) CUDA_TRY(h, cudaStreamWaitEvent(pl.side, h->fork, 0));
+            Params p = h->params;
+            p.t0 = h->t_done;
+            p.n_steps = now;
+            p.groups = h->d_pgroups + pl.pg_off;
+            p.n_groups = pl.pg_cnt;
+            p.n_work = pl.n_work;
+            p.work_counter = h->d_work + pl.policy;
+            p.tabcache_off = (uint32_t)pl.tabcache_off;
+            // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
+            CUDA_TRY(h, cudaFuncSetAttribute(pl.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_block));
+            pl.kernel<<<pl.grid, pl.warps_per_block * 32, pl.smem_block, ls>>>(p);
+            CUDA_TRY(h, cudaGetLastError());
+            if (pl.side) CUDA_TRY(h, cudaEventRecord(pl.done, pl.side));
+        }
+        for (const PolicyLaunch& pl : h->launches)
+            if (pl.side) CUDA_TRY(h, cudaStreamWaitEvent(st, pl.done, 0));
         h->t_done += now;
         left -= now;
     }
@@ -694,12 +785,13 @@ extern "C" int32_t fcsim_steps_done(const fcsim_t* h) { return h ? h->t_done : -
 
 extern "C" int fcsim_get_launch_info(const fcsim_t* h, fcsim_launch_info* out) {
     if (!h || !out) return FCSIM_EINVAL;
-    out->grid = h->grid;
-    out->block = h->L.warps_per_block * 32;
-    out->warps_per_block = h->L.warps_per_block;
-    out->blocks_per_sm = h->blocks_per_sm;
+    const PolicyLaunch& pl = h->launches[h->main_launch];  // the policy with the most replicas
+    out->grid = pl.grid;
+    out->block = pl.warps_per_block * 32;
+    out->warps_per_block = pl.warps_per_block;
+    out->blocks_per_sm = pl.blocks_per_sm;
     out->sm_count = h->sm_count;
-    out->smem_per_block = (int32_t)h->smem_block;
+    out->smem_per_block = (int32_t)pl.smem_block;
     out->smem_per_warp = (int32_t)h->L.smem_per_warp;
     out->max_steps_per_launch = max_steps_per_launch(h);
     return FCSIM_OK;

@@ -68,12 +68,14 @@ struct DevGroup {
     int32_t bclass_off;   // Algorithm 1: index of the group's per-class budgets in Params::bclass
     int32_t mc_worst;     // MC benchmark: project with the class's longest output length
     int32_t keep;         // 1 = an evicted request keeps its generated tokens as prompt: (l, o) <- (l + j, o - j)
+    int32_t wfirst;       // index of the group's first replica among the work items of its policy's launch
 };
 
 struct Params {
     int32_t M, K, Qcap, Acap, RC, S, Apad;  // RC, Apad: padded storage sizes of the two rings
     uint32_t key0, key1;
-    int32_t n_classes, n_groups, n_replicas;
+    int32_t n_classes, n_groups, n_replicas;  // n_groups: entries of `groups`
+    int32_t n_work;               // replicas this launch advances (those of the groups in `groups`)
     int32_t trace_stride, n_rec, hist_bins, hist_shift, complog_cap;
     int32_t t0, n_steps;
     const uint32_t* pool;         // all thresholds
@@ -87,7 +89,7 @@ struct Params {
                                   // memory; 0 = records are kept in registers and stored with plain stores
     const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
     const DevArrivals* arrivals;
-    const DevGroup* groups;
+    const DevGroup* groups;       // the groups of this launch's policy, in replica order
     unsigned char* workspace;     // [R] records of ws_stride bytes
     unsigned long long ws_stride;
     long long* counters;          // [R][C_COUNT]
@@ -248,13 +250,20 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define HROW(i) hrow[(i)]
 #endif
 
-// kExt: compiled with the per-class activation of Algorithm 1 (policy 4) and the future-memory test of the
-// MC benchmark (policy 5); the variant without them is used when no group asks for either, so that the
-// common policies do not carry their code.
-// kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80 with a
-// few spilled words).  The host picks 6 when the shared memory of six CTAs fits the SM, else 5.
-template <bool kExt, int kMinCtas>
+// One launch advances the replicas of the groups that share one policy; a configuration with several
+// policies is run as several launches that the host issues side by side.
+// kPol: the policy, a compile-time constant: the slot loop is one long chain of short warp-uniform decisions,
+// and every test of the policy that the compiler resolves shortens it (and frees the registers of the state
+// that only other policies keep).
+// kRec: what is recorded per slot: 0 = no trace and no completion log, 1 = trace only, 2 = whatever the
+// parameters say (decided at run time).
+// kExt (= kPol >= 4): the per-class activation of Algorithm 1 (policy 4) and the future-memory test of the MC
+// benchmark (policy 5) use extra per-warp state (class counts, projection words).
+// kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80).  The host
+// asks the occupancy calculator about both.
+template <int kPol, int kMinCtas, int kRec>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
+    constexpr bool kExt = kPol >= 4;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // the table descriptors of the length laws are read for every generated arrival: the host reserves room
     // for a copy behind the warps' slices when that does not cost a resident CTA
@@ -286,28 +295,29 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 
     for (;;) {
         // ------------------------------------------------------------------ next replica
-        unsigned int r = 0;
-        if (lane == 0) r = atomicAdd(p.work_counter, 1u);
-        r = __shfl_sync(FULL, r, 0);
-        if (r >= (unsigned)p.n_replicas) break;
+        unsigned int wi = 0;  // work item: the wi-th replica of this policy
+        if (lane == 0) wi = atomicAdd(p.work_counter, 1u);
+        wi = __shfl_sync(FULL, wi, 0);
+        if (wi >= (unsigned)p.n_work) break;
 
         int gi = 0;
         {
             int lo = 0, hi = p.n_groups - 1;
-            while (lo < hi) {  // last group whose first replica is <= r
+            while (lo < hi) {  // last group whose first work item is <= wi
                 const int mid = (lo + hi + 1) >> 1;
-                if (p.groups[mid].first <= (int)r) lo = mid; else hi = mid - 1;
+                if (p.groups[mid].wfirst <= (int)wi) lo = mid; else hi = mid - 1;
             }
             gi = lo;
         }
         const DevGroup grp = p.groups[gi];
+        const unsigned int r = (unsigned)grp.first + (wi - (unsigned)grp.wfirst);  // the replica's index
         const DevArrivals* arrp = p.arrivals + grp.arrivals_id;
         const DevTable cnt0 = arrp->count[0];
         const DevTable cnt1 = arrp->count[1];
         const uint32_t thr0 = arrp->thr[0], thr1 = arrp->thr[1];
         const bool two_state = arrp->n_states == 2;
         const uint32_t rid = grp.rng_base + (r - (unsigned)grp.first);
-        const int policy = grp.policy;
+        constexpr int policy = kPol;
         const int chunk = grp.chunk;
         const int admit_limit = grp.admit_limit;
 
@@ -366,19 +376,20 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         const int t_end = p.t0 + p.n_steps;
 
         // trace bookkeeping: lane (rec & 31) holds record rec until its block of 32 is flushed
-        const int stride = p.trace_stride;
-        int rec = stride > 0 ? t / stride : 0;
-        int cd = stride > 0 ? stride - (t % stride) : 0;
+        const int stride = (kRec == 0) ? 0 : p.trace_stride;
+        const bool tracing = (kRec == 1) || (kRec == 2 && stride > 0);
+        int rec = tracing ? t / stride : 0;
+        int cd = tracing ? stride - (t % stride) : 0;
         const int rec_lo = rec;
         int tr_u = 0, tr_q = 0;
         // staged variant: records go to shared memory (two buffers of 32) and every full block of 32 leaves
         // with one 256-byte bulk copy issued by lane 0, when the row's address allows it
         int2* tstage = reinterpret_cast<int2*>(my + p.tstage_off);
-        const bool staged = p.tstage_off != 0 && stride > 0 &&
+        const bool staged = p.tstage_off != 0 && tracing &&
                             ((reinterpret_cast<uintptr_t>(p.trace + (size_t)r * p.n_rec) & 15u) == 0);
-        int2* trow = p.trace ? p.trace + (size_t)r * p.n_rec : nullptr;
+        int2* trow = (kRec != 0 && p.trace) ? p.trace + (size_t)r * p.n_rec : nullptr;
         int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
-        int2* lrow = p.complog ? p.complog + (size_t)r * p.complog_cap : nullptr;
+        int2* lrow = (kRec == 2 && p.complog) ? p.complog + (size_t)r * p.complog_cap : nullptr;
 
         // Squeeze the completed entries out of the active range: survivors slide towards the queue
         // boundary (right-to-left pass), the head advances, the queue is not touched.
@@ -577,7 +588,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         rebuild_minima();
                         squeeze = false;
                     }
-                    if ((kExt && policy == 4)) {
+                    if constexpr (policy == 4) {
                         // Algorithm 1: for every class k, up to b_k waiting requests of that class, oldest first.
                         // The pick leaves the middle of the queue: the entries ahead of it move one place
                         // towards the tail and the pick takes the freed place next to the active range.
@@ -636,7 +647,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         if (storage_hit) { CADD(C_ACAP_BLOCKED, 1); status |= 1u; }
                         q_e = 0;
                         break;
-                    }
+                    } else {
                     while (a < cap && nQ > 0) {
                         if (nP == Acap) {
                             if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room
@@ -747,6 +758,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         CADD(C_PREFILL_TOKENS, g);
                     }
                     if (!squeeze) break;
+                    }
                 }
                 if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
 
@@ -956,7 +968,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 
                 // ---- record
                 maxQ = max(maxQ, nQ);
-                if (stride > 0 && --cd == 0) {
+                if (tracing && --cd == 0) {
                     cd = stride;
                     if (staged) {
                         if (lane == 0) tstage[rec & 63] = make_int2(G, nQ);
@@ -987,7 +999,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         }  // while t < t_end
 
         // ------------------------------------------------------------------ flush, final extras, spill
-        if (stride > 0 && (rec & 31) != 0) {
+        if (tracing && (rec & 31) != 0) {
             const int b0 = rec & ~31;
             if (staged) {
                 __syncwarp();
