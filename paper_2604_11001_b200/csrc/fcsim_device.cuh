@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 
         // per-launch partial sums of the quantities touched every slot
         unsigned long long sumU = 0;
-        uint32_t sumN = 0, tokgen = 0, arrived = 0, dropped = 0;
+        uint32_t sumN = 0, tokgen = 0, arrived = 0, accepted = 0;
         int maxU = 0, maxQ = 0;
         int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
         uint64_t q_e = 0;  // the queue head's entry when known, else 0 (saves shared-memory reads in blocked slots)
@@ -496,32 +496,34 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 }
             }
             __syncwarp();
-            const uint32_t packed = (uint32_t)n | ((uint32_t)Bt << 8);
-            int sp = 0;  // staged arrivals consumed so far
+            // A slot asks for its count only when it has arrivals AND the waiting room has a place: bit k of
+            // nzmask says whether slot k has arrivals, lane k holds the count and where its arrivals are staged.
+            // Arrivals that find the room full are dropped without being looked at; their number is the
+            // difference between the batch's total and the accepted ones.
+            const uint32_t nzmask = __ballot_sync(FULL, n > 0);
+            const uint32_t btmask = __ballot_sync(FULL, Bt > (int)(grp.b_fp >> 16));  // slots whose B_t is rounded up
+            const uint32_t packed = (uint32_t)n | ((uint32_t)excl << 8);
+            arrived += N;
 
             // -------------------------------------------------------------- the slots of the batch
             for (int k = 0; k < L; ++k) {
                 ++t;
-                const uint32_t info = __shfl_sync(FULL, packed, k);
-                const int n_t = (int)(info & 0xffu);
-                const int B_t = (int)(info >> 8);
+                const int B_t = (int)(grp.b_fp >> 16) + (int)((btmask >> k) & 1u);
 
                 // ---- arrivals join the queue tail; a full waiting room drops the rest
-                if (n_t > 0) {
-                    const int acc = min(n_t, max(0, Qcap - nQ));
-                    if (acc > 0) {
-                        const int tail = WR(head + nP + nQ);
-                        for (int i = lane; i < acc; i += 32) {
-                            const uint64_t e = STAGE(sp + i);
-                            RING(WR(tail + i)) = e;
-                            if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
-                        }
-                        nQ += acc;
-                        __syncwarp();
+                if (((nzmask >> k) & 1u) && nQ < Qcap) {
+                    const uint32_t info = __shfl_sync(FULL, packed, k);
+                    const int sp = (int)(info >> 8);  // where the slot's arrivals are staged
+                    const int acc = min((int)(info & 0xffu), Qcap - nQ);
+                    const int tail = WR(head + nP + nQ);
+                    for (int i = lane; i < acc; i += 32) {
+                        const uint64_t e = STAGE(sp + i);
+                        RING(WR(tail + i)) = e;
+                        if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
                     }
-                    sp += n_t;
-                    arrived += n_t;
-                    dropped += n_t - acc;
+                    nQ += acc;
+                    accepted += acc;
+                    __syncwarp();
                 }
 
                 // ---- usage the slot would reach, token room
@@ -1029,7 +1031,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         CADD(C_SUM_N, sumN);
         CADD(C_TOKENS_GENERATED, tokgen);
         CADD(C_ARRIVED, arrived);
-        CADD(C_DROPPED, dropped);
+        CADD(C_DROPPED, arrived - accepted);
         CADD(C_COMPLETED, completed);
         CADD(C_SUM_LAT, warp_sum64((long long)acc_lat));
         CADD(C_SUM_W_COMPLETED, warp_sum64((long long)acc_w));
