@@ -20,6 +20,7 @@ namespace {
 constexpr size_t kSmemBudget = 227 * 1024;   // shared memory one CTA may opt in to
 constexpr int kMaxStepsPerLaunch = 32768;    // keeps the 32-bit per-launch partial sums exact
 constexpr long long kTargetWorkPerLaunch = 1LL << 31;  // replica-steps per launch (bounds launch time)
+constexpr uint64_t kGuideMaxRecords = 16384;  // per table: 256 KB of 16-byte records
 constexpr int kStatsChunk = 256;             // replicas reduced by one block before it touches the group row
 
 struct Layout {
@@ -293,7 +294,7 @@ struct fcsim {
     fcsim_buffers buf;
     Params params;
     uint32_t* d_pool = nullptr;
-    unsigned short* d_gpool = nullptr;
+    uint4* d_gpool = nullptr;
     int32_t* d_bclass = nullptr;
     std::vector<PolicyLaunch> launches;  // most expensive policy first
     int main_launch = 0;                 // the launch with the most replicas (reported by fcsim_get_launch_info)
@@ -337,7 +338,28 @@ extern "C" int fcsim_query_sizes(const fcsim_config* cfg, fcsim_sizes* out) {
 
 static int upload_tables(fcsim* h, const fcsim_config* c) {
     std::vector<uint32_t> pool;
-    std::vector<unsigned short> gpool(2, 0);  // offset 0 is never a guide
+    std::vector<uint4> gpool;
+    // Guide of a table (see guide_bucket in the device code): one record per bucket of the 32-bit range.  The
+    // bucket scheme (g, J) is the candidate that leaves the least probability mass to the fall-back search,
+    // within kGuideMaxRecords per table; equal buckets (J = 0) suit flat laws, halving buckets (J > 0) suit
+    // laws with a long upper tail.
+    auto bucket_range = [](uint32_t g, uint32_t J, uint32_t j, uint32_t m, uint32_t* ulo, uint32_t* uhi) {
+        // bucket (j, m) holds the v = ~u with clz(v) == j (>= J for j == J) and mantissa m; false if it is empty
+        const uint32_t sh = j + (j < J ? 1u : 0u);
+        const uint32_t rem = 32u - sh;  // bits of v below the consumed ones
+        uint64_t vlo, vhi;
+        if (rem >= g) {
+            vlo = (uint64_t)m << (rem - g);
+            vhi = vlo | ((1ull << (rem - g)) - 1ull);
+        } else {
+            if (m & ((1u << (g - rem)) - 1u)) return false;
+            vlo = vhi = m >> (g - rem);
+        }
+        if (j < J) { vlo |= 1ull << rem; vhi |= 1ull << rem; }
+        *ulo = ~(uint32_t)vhi;
+        *uhi = ~(uint32_t)vlo;
+        return true;
+    };
     auto add = [&](const fcsim_table& t) {
         DevTable d;
         d.off = (uint32_t)pool.size();
@@ -345,20 +367,44 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         d.vmin = t.vmin;
         d.guide = 0;
         pool.insert(pool.end(), t.cdf, t.cdf + t.n);
-        if (t.n >= 16) {
-            // guide[b] = first k < n-1 with cdf[k] > (b << shift), else n-1; guide[2^bits] = n-1
-            // about two table entries per bucket, so that the search after the guide is one or two probes
-            uint32_t bits = 4;
-            while (bits < 12 && (2u << bits) < t.n) ++bits;
-            const uint32_t shift = 32 - bits;
-            d.guide = (bits << 27) | (uint32_t)gpool.size();
-            uint32_t k = 0;
-            for (uint32_t b = 0; b < (1u << bits); ++b) {
-                const uint32_t edge = b << shift;
-                while (k < t.n - 1 && t.cdf[k] <= edge) ++k;
-                gpool.push_back((unsigned short)k);
+        if (t.n >= 2) {
+            const uint32_t* thr_end = t.cdf + (t.n - 1);  // real thresholds: cdf[0 .. n-2]
+            auto first_above = [&](uint32_t x) { return (uint32_t)(std::upper_bound(t.cdf, thr_end, x) - t.cdf); };
+            double best_mass = 2.0;
+            uint32_t best_g = 0, best_J = 0;
+            for (uint32_t J = 0; J <= 20; J += 4) {
+                for (uint32_t g = 4; g <= 14; ++g) {
+                    const uint64_t records = (uint64_t)(J + 1) << g;
+                    if (records > kGuideMaxRecords) break;
+                    if (J > 0 && g > 10) break;
+                    double mass = 0.0;
+                    for (uint32_t j = 0; j <= J; ++j)
+                        for (uint32_t m = 0; m < (1u << g); ++m) {
+                            uint32_t ulo, uhi;
+                            if (!bucket_range(g, J, j, m, &ulo, &uhi)) continue;
+                            const uint32_t k3 = first_above(ulo) + 2;  // third threshold above the bucket's low end
+                            if (k3 < t.n - 1 && t.cdf[k3] <= uhi) mass += (double)uhi - (double)std::max(t.cdf[k3], ulo) + 1.0;
+                        }
+                    mass /= 4294967296.0;
+                    // a larger guide must buy a clearly smaller fall-back mass, and 1e-4 is small enough
+                    if (best_mass > 1.5 || (best_mass > 1e-4 && mass < best_mass * 0.7)) { best_mass = mass; best_g = g; best_J = J; }
+                    if (mass <= 1e-4) break;
+                }
             }
-            gpool.push_back((unsigned short)(t.n - 1));
+            d.guide = (best_g << 27) | (best_J << 22) | (uint32_t)gpool.size();
+            for (uint32_t j = 0; j <= best_J; ++j)
+                for (uint32_t m = 0; m < (1u << best_g); ++m) {
+                    uint32_t ulo = 0, uhi = 0;
+                    uint4 rec = make_uint4(t.n - 1, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+                    if (bucket_range(best_g, best_J, j, m, &ulo, &uhi)) {
+                        const uint32_t k0 = first_above(ulo);
+                        rec.x = k0;
+                        if (k0 + 0 < t.n - 1) rec.y = t.cdf[k0];
+                        if (k0 + 1 < t.n - 1) rec.z = t.cdf[k0 + 1];
+                        if (k0 + 2 < t.n - 1) rec.w = t.cdf[k0 + 2];
+                    }
+                    gpool.push_back(rec);
+                }
         }
         return d;
     };
@@ -409,8 +455,10 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
     }
     CUDA_TRY(h, cudaMalloc(&h->d_bclass, bclass.size() * sizeof(int32_t)));
     CUDA_TRY(h, cudaMemcpy(h->d_bclass, bclass.data(), bclass.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
-    CUDA_TRY(h, cudaMalloc(&h->d_gpool, gpool.size() * sizeof(unsigned short)));
-    CUDA_TRY(h, cudaMemcpy(h->d_gpool, gpool.data(), gpool.size() * sizeof(unsigned short), cudaMemcpyHostToDevice));
+    if (gpool.empty()) gpool.push_back(make_uint4(0, 0, 0, 0));
+    if (gpool.size() > (size_t)0x3fffff) return FCSIM_ECAP;  // a guide's first record is a 22-bit index
+    CUDA_TRY(h, cudaMalloc(&h->d_gpool, gpool.size() * sizeof(uint4)));
+    CUDA_TRY(h, cudaMemcpy(h->d_gpool, gpool.data(), gpool.size() * sizeof(uint4), cudaMemcpyHostToDevice));
     CUDA_TRY(h, cudaMalloc(&h->d_pool, pool.size() * sizeof(uint32_t)));
     CUDA_TRY(h, cudaMalloc(&h->d_tables, tables.size() * sizeof(DevTable)));
     CUDA_TRY(h, cudaMalloc(&h->d_arrivals, arrs.size() * sizeof(DevArrivals)));

@@ -48,7 +48,7 @@ struct DevTable {
     uint32_t off;  // first threshold in the pool
     uint32_t n;
     int32_t vmin;
-    uint32_t guide;  // bits 27..31: log2 of the guide size (0 = no guide); bits 0..26: offset in the guide pool
+    uint32_t guide;  // 0 = none; else bits 27..31: g (mantissa bits), 22..26: J (levels), 0..21: first record in the guide pool
 };
 struct DevArrivals {
     DevTable count[2];
@@ -79,7 +79,7 @@ struct Params {
     int32_t trace_stride, n_rec, hist_bins, hist_shift, complog_cap;
     int32_t t0, n_steps;
     const uint32_t* pool;         // all thresholds
-    const unsigned short* gpool;  // guide tables: for bucket b of the top bits of u, the first candidate index
+    const uint4* gpool;           // guide records {k0, thresholds k0, k0+1, k0+2}, one per bucket of u
     const int32_t* bclass;        // per-class budgets b_k of the Algorithm-1 groups
     uint32_t qcnt_off;            // byte offset of the per-class queue counts in a warp's shared memory (0 = none)
     uint32_t tabcache_off;        // byte offset in the CTA's shared memory of a copy of `tables` (0 = none)
@@ -118,20 +118,39 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     o0 = c0; o1 = c1; o2 = c2; o3 = c3;
 }
 
-// vmin + (first k < n-1 with thresholds[k] > u, else n-1).  A guide table indexed by the top bits of u
-// brackets the answer (entry b = first index whose threshold exceeds b << shift), so the binary search
-// runs over a few entries instead of the whole table.
-__device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, const unsigned short* __restrict__ gpool,
+// Inverse-CDF lookup: vmin + (first k < n-1 with thresholds[k] > u, else n-1).
+// A table with a guide answers with ONE 16-byte load in all but rare cases.  The 32-bit range of u is cut into
+// buckets; the record of a bucket holds k0, the first index whose threshold exceeds the bucket's lowest u, and the
+// thresholds k0, k0+1, k0+2 (0xffffffff where there is none), so the answer is k0 plus the number of those that
+// are <= u.  Only when all three are (a bucket with more than three thresholds, or the very top of the range)
+// does a binary search over the thresholds from k0+3 finish the job.
+// Buckets: with v = ~u and j = min(clz(v), J), bucket (j, m) takes the g bits m that follow the leading one of
+// v (for j == J: the g bits after J leading zeros).  J = 0 gives 2^g equal buckets; J > 0 halves the bucket
+// width with every leading one of u, which keeps the long thin upper tail of a geometric or lognormal law at a
+// few thresholds per bucket.  The host picks (g, J) per table.
+__device__ __forceinline__ uint32_t guide_bucket(uint32_t guide, uint32_t u) {
+    const uint32_t g = guide >> 27, J = (guide >> 22) & 31u;
+    const uint32_t v = ~u;
+    const uint32_t j = min((uint32_t)__clz((int)v), J);
+    const uint32_t sh = j + (j < J ? 1u : 0u);  // bits before the mantissa; <= 31 because J <= 30
+    return (guide & 0x3fffffu) + (j << g) + ((v << sh) >> (32u - g));
+}
+__device__ __forceinline__ int guide_finish(const uint32_t* __restrict__ cdf, uint32_t n, uint4 rec, uint32_t u) {
+    uint32_t k = rec.x + (rec.y <= u ? 1u : 0u) + (rec.z <= u ? 1u : 0u) + (rec.w <= u ? 1u : 0u);
+    if (rec.w <= u) {
+        uint32_t hi = n - 1;
+        while (k < hi) {
+            const uint32_t mid = (k + hi) >> 1;
+            if (__ldg(cdf + mid) > u) hi = mid; else k = mid + 1;
+        }
+    }
+    return (int)min(k, n - 1);
+}
+__device__ __forceinline__ int sample_table(const uint32_t* __restrict__ pool, const uint4* __restrict__ gpool,
                                             const DevTable tb, uint32_t u) {
     const uint32_t* __restrict__ cdf = pool + tb.off;
+    if (tb.guide >> 27) return tb.vmin + guide_finish(cdf, tb.n, __ldg(gpool + guide_bucket(tb.guide, u)), u);
     uint32_t lo = 0, hi = tb.n - 1;
-    const uint32_t gbits = tb.guide >> 27;
-    if (gbits) {
-        const unsigned short* __restrict__ g = gpool + (tb.guide & 0x7ffffffu);
-        const uint32_t b = u >> (32u - gbits);
-        lo = __ldg(g + b);
-        hi = __ldg(g + b + 1);
-    }
     while (lo < hi) {
         const uint32_t mid = (lo + hi) >> 1;
         if (__ldg(cdf + mid) > u) hi = mid; else lo = mid + 1;
@@ -154,35 +173,20 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// Two independent table searches (prompt and decode length of one arrival) advanced in the same loop, so
-// that their dependent global loads overlap instead of running one chain after the other.
-__device__ __forceinline__ void sample_pair(const uint32_t* __restrict__ pool, const unsigned short* __restrict__ gpool,
+// Two independent lookups (prompt and decode length of one arrival): both records are requested before either
+// is used, so that their round trips to the L2 overlap.
+__device__ __forceinline__ void sample_pair(const uint32_t* __restrict__ pool, const uint4* __restrict__ gpool,
                                             const DevTable ta, uint32_t ua, const DevTable tb, uint32_t ub, int& va,
                                             int& vb) {
-    const uint32_t* __restrict__ ca = pool + ta.off;
-    const uint32_t* __restrict__ cb = pool + tb.off;
-    uint32_t loa = 0, hia = ta.n - 1, lob = 0, hib = tb.n - 1;
-    const uint32_t ga = ta.guide >> 27, gb = tb.guide >> 27;
-    if (ga) {
-        const unsigned short* __restrict__ g = gpool + (ta.guide & 0x7ffffffu);
-        const uint32_t b = ua >> (32u - ga);
-        loa = __ldg(g + b);
-        hia = __ldg(g + b + 1);
+    if ((ta.guide >> 27) && (tb.guide >> 27)) {
+        const uint4 ra = __ldg(gpool + guide_bucket(ta.guide, ua));
+        const uint4 rb = __ldg(gpool + guide_bucket(tb.guide, ub));
+        va = ta.vmin + guide_finish(pool + ta.off, ta.n, ra, ua);
+        vb = tb.vmin + guide_finish(pool + tb.off, tb.n, rb, ub);
+    } else {
+        va = sample_table(pool, gpool, ta, ua);
+        vb = sample_table(pool, gpool, tb, ub);
     }
-    if (gb) {
-        const unsigned short* __restrict__ g = gpool + (tb.guide & 0x7ffffffu);
-        const uint32_t b = ub >> (32u - gb);
-        lob = __ldg(g + b);
-        hib = __ldg(g + b + 1);
-    }
-    while (loa < hia || lob < hib) {
-        const uint32_t ma = (loa + hia) >> 1, mb = (lob + hib) >> 1;
-        const uint32_t xa = __ldg(ca + ma), xb = __ldg(cb + mb);  // both probes in flight together (in range always)
-        if (loa < hia) { if (xa > ua) hia = ma; else loa = ma + 1; }
-        if (lob < hib) { if (xb > ub) hib = mb; else lob = mb + 1; }
-    }
-    va = ta.vmin + (int)loa;
-    vb = tb.vmin + (int)lob;
 }
 
 __device__ __forceinline__ uint32_t lanemask_lt() {
