@@ -34,7 +34,6 @@ constexpr int kHeaderWords = 16;  // per-replica scalar state kept in the worksp
 constexpr uint32_t kNoFin = 0xFFFFFFFFu;
 constexpr uint32_t kPrefillBit = 0x80000000u;
 constexpr uint32_t kDead = 0u;        // state word of a completed entry awaiting removal
-constexpr int kCompactAt = 32;        // completed entries tolerated inside the active range
 
 enum CounterIdx {
     C_STEPS_DONE = 0, C_STATUS, C_ARRIVED, C_DROPPED, C_ADMITTED, C_COMPLETED, C_EVICTIONS,
@@ -268,6 +267,11 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 template <int kPol, int kMinCtas, int kRec>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     constexpr bool kExt = kPol >= 4;
+    // Completed entries tolerated inside the active range before they are squeezed out (they always are when the
+    // storage runs out).  The whole-prompt policies touch the range only where a request finishes, so removal
+    // as late as possible measured fastest; the policies that walk the range (chunked prefills, Algorithm 1's
+    // storage check, the MC projections) want it short.
+    constexpr int kCompactAt = (kPol <= 1 || kPol == 3) ? 256 : 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // the table descriptors of the length laws are read for every generated arrival: the host reserves room
     // for a copy behind the warps' slices when that does not cost a resident CTA
