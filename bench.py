@@ -29,12 +29,12 @@ if ROOT not in sys.path:
 METRIC = "simulated replica-steps/s"
 UNIT = "replica-steps/s"
 
-# Executed warp-instructions per replica-step of the step kernel in the timed regime of each preset,
-# from the committed ncu captures (profiles/): smsp__inst_executed.sum / (replicas x slots) of one launch.
-# None = not captured for the current kernel.
-INST_PER_REPLICA_STEP = {1: 270.8, 2: 311.7, 3: 357.5, 4: 446.9, 5: 258.4, 6: 2303.4}
+# Executed warp-instructions per replica-step of the step kernels in the timed regime of each preset, from the
+# committed ncu captures (profiles/): smsp__inst_executed.sum over the launches of one bench step (one kernel per
+# policy present) / (replicas x slots).  None = not captured for the current kernels.
+INST_PER_REPLICA_STEP = {1: 238.3, 2: 259.4, 3: 297.9, 4: 396.6, 5: 192.4, 6: 2004.9}
 # DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
-DRAM_BYTES_PER_REPLICA_STEP = {1: 29.1, 2: 22.9, 3: 17.8, 4: 10.0, 5: 7.9, 6: 79.6}
+DRAM_BYTES_PER_REPLICA_STEP = {1: 31.2, 2: 15.5, 3: 17.9, 4: 9.0, 5: 7.0, 6: 58.8}
 
 DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000, 6: 500}
 NAMES = {1: "cfg1-tiny-flow", 2: "cfg2-policy-comparison", 3: "cfg3-stability-sweep", 4: "cfg4-heavy-tail",
@@ -246,7 +246,8 @@ def main():
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         ms_total = float(tmax.item())
     value = world * R * chunk * args.steps / (ms_total * 1e-3)
-    launches_per_step = -(-chunk // info["max_steps_per_launch"])
+    n_policies = len({g.policy for g in cfg.groups})   # one kernel per policy, side by side on forked streams
+    launches_per_step = -(-chunk // info["max_steps_per_launch"]) * n_policies
 
     # sanity of the timed state: the counters must show the work was done
     counters, summary = sim.stats(stream)
@@ -294,9 +295,11 @@ def main():
     peak_ginst = info["sm_count"] * 4 * sm_mhz * 1e6 / 1e9       # warp-instructions/s the schedulers can issue
     ipr = INST_PER_REPLICA_STEP.get(args.workload)
     dbr = DRAM_BYTES_PER_REPLICA_STEP.get(args.workload)
-    kernel_ms = statistics.mean(per_step) / launches_per_step
+    kernel_ms = statistics.mean(per_step) / (launches_per_step // n_policies)
     roofline = {
-        "bound": "alu", "kernel": "fcsim_step_kernel",
+        "bound": "alu",
+        "kernel": "fcsim_step_kernel<policy, ctas, rec>: %d concurrent launch(es) per step, one per policy; figures "
+                  "are sums over them" % n_policies,
         "achieved": (ipr * value / world / 1e9) if ipr else None,
         "peak": peak_ginst, "unit": "Gwarp-inst/s",
         "frac": (ipr * value / world / 1e9 / peak_ginst) if ipr else None,
@@ -304,7 +307,7 @@ def main():
         "inst_per_replica_step": ipr,
         "peak_basis": "%d SMs x 4 schedulers x %.0f MHz (median SM clock sampled during the timed region)"
                       % (info["sm_count"], sm_mhz),
-        "kernel_ms_per_launch": kernel_ms, "launches_per_step": launches_per_step,
+        "kernel_ms_per_launch": kernel_ms, "launches_per_step": launches_per_step, "policies": n_policies,
         "hbm_peak_gbs": peaks.get("hbm_gbs"), "hbm_peak_kind": peak_kind,
     }
     if cfg.trace_stride > 0:

@@ -177,7 +177,8 @@ typedef struct {
     size_t workspace, counters, trace, hist, complog, scratch;
 } fcsim_sizes;
 
-/* Launch geometry chosen for a handle (for reporting). */
+/* Launch geometry chosen for a handle (for reporting).  A configuration whose groups use several policies is
+ * advanced by one kernel per policy; the figures are those of the policy with the most replicas. */
 typedef struct {
     int32_t grid, block, warps_per_block, blocks_per_sm, sm_count;
     int32_t smem_per_block, smem_per_warp, max_steps_per_launch;
@@ -194,7 +195,11 @@ int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* device_buffers, f
 
 /* Advances every replica by n_steps slots (steps_done + n_steps <= T_max, else FCSIM_ERANGE).
  * Asynchronous on `cuda_stream` (a cudaStream_t; NULL = default stream).  Resumable: run(a) then run(b)
- * gives bit for bit the state and outputs of run(a+b).  Long runs are split into several launches. */
+ * gives bit for bit the state and outputs of run(a+b).  Long runs are split into several launches.
+ * The groups of each policy are advanced by a kernel compiled for that policy.  With several policies the
+ * kernels run side by side: the first on `cuda_stream`, the others on streams owned by the handle that are
+ * forked from and joined back to `cuda_stream` with events, so work enqueued on `cuda_stream` after the call
+ * sees all of them finished. */
 int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream);
 
 /* Reduces counters and histograms per group on the device, then synchronises `cuda_stream` and copies:

@@ -267,3 +267,38 @@ def test_mc_many_finishers_in_one_slot():
         if M == 330:
             assert (c[:, orc.CIDX["gate_blocked_steps"]] > 50).all()
         assert_same(cfg, run_gpu(cfg, pieces=[100, 200]), ref, 300, f"MC finishers M={M} worst={mode}")
+
+
+def test_policies_interleaved_over_groups_on_a_side_stream():
+    # every policy's kernel walks a work list made of several non-adjacent groups of unequal size; the call is
+    # made on a stream other than the default one, in resumed pieces, and the kernels of the policies run side
+    # by side on streams of the handle
+    import dataclasses
+    import torch
+    from paper_2604_11001_b200 import binding as fb
+    base = wl.random_medium_config(3, n_replicas=1)
+    proto = {g.policy: g for seed in (3, 4, 5, 6) for g in wl.random_medium_config(seed).groups}
+    order = [1, 0, 3, 1, 2, 0, 0, 5, 1, 4, 2, 0]
+    sizes = [3, 1, 2, 5, 1, 4, 2, 2, 1, 3, 2, 6]
+    groups, rid = [], 0
+    for pol, n in zip(order, sizes):
+        if pol not in proto:
+            continue
+        groups.append(dataclasses.replace(proto[pol], n_replicas=n, rng_replica_base=rid,
+                                          b_class=(2, 1, 1, 1)[:base.n_classes]))
+        rid += n
+    cfg = base.with_(groups=tuple(groups), T_max=1200, Acap=200, Qcap=40, complog_cap=300)
+    assert len({g.policy for g in cfg.groups}) >= 4
+    ref = orc.run(cfg, threads=8)
+    sim = fb.Simulation(cfg)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for piece in (1, 499, 700):
+            sim.run(piece, side)
+        counters, summary = sim.stats(side)
+    gpu = {"counters": counters, "summary": summary}
+    for name in ("trace", "hist", "complog"):
+        v = getattr(sim, name)()
+        gpu[name] = None if v is None else v.cpu().numpy()
+    sim.close()
+    assert_same(cfg, gpu, ref, 1200, "interleaved policies")
