@@ -321,7 +321,11 @@ def main():
         "config": {"workload": NAMES[args.workload], "replicas_per_gpu": R, "slots_per_step": chunk,
                    "warm_slots": args.warmup * chunk, "groups": len(cfg.groups), "M": cfg.M, "K": cfg.K,
                    "Qcap": cfg.Qcap, "Acap": cfg.Acap,
-                   "l2": "replica state %.0f MB exceeds the 126 MB L2; no explicit flush" % (sizes["workspace"] / 1e6),
+                   "l2": ("replica state %.0f MB exceeds the 126 MB L2; no explicit flush" % (sizes["workspace"] / 1e6)
+                          if sizes["workspace"] > 126e6 else
+                          "replica state %.0f MB fits the 126 MB L2 (small preset); its %.0f MB of per-slot outputs do "
+                          "not; no explicit flush" % (sizes["workspace"] / 1e6,
+                                                     (sizes["trace"] + sizes["complog"] + sizes["hist"]) / 1e6)),
                    "launch": info, "parallelism": "replicas only, %d per GPU" % R},
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_step,
         "roofline": roofline, "cpu_baseline": cpu_baseline,

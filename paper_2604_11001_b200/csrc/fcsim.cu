@@ -24,7 +24,9 @@ constexpr uint64_t kGuideMaxRecords = 16384;  // per table: 256 KB of 16-byte re
 constexpr int kStatsChunk = 256;             // replicas reduced by one block before it touches the group row
 
 struct Layout {
-    int RC, Apad, S;
+    int Apad, S;
+    uint32_t QC;                                // queue ring in global memory: entries (a power of two)
+    size_t gq_off, qwin_off;                    // queue ring in the workspace record; queue window in shared memory
     size_t ws_stride, smem_per_warp, qcnt_off;  // qcnt_off: per-class queue counts (Algorithm 1), 0 = unused
     size_t tstage_off;                          // trace staging buffers, 0 = unused
     size_t state_bytes;                         // ring + state words (+ projection words) saved between launches
@@ -99,14 +101,19 @@ int plan(const fcsim_config* c, Layout* L) {
 
     const long long rc = (long long)c->Qcap + c->Acap;  // evictions may push the queue past Qcap
     if (rc > (1 << 20)) return FCSIM_ECAP;
-    L->RC = (int)align_up((size_t)rc, 2);
+    L->QC = 64;
+    while ((long long)L->QC < rc) L->QC <<= 1;
     L->Apad = (int)align_up((size_t)c->Acap, 4);
     L->S = (int)align_up((size_t)std::max(128, max_count), 2);
     // the MC benchmark keeps one more word per active entry (projected usage in its last slot), saved with the state
-    L->state_bytes = (size_t)L->RC * 8 + (size_t)L->Apad * 4 * (any_mc ? 2 : 1);
+    L->state_bytes = (size_t)L->Apad * 8 + (size_t)L->Apad * 4 * (any_mc ? 2 : 1);
     L->has_v = any_mc ? 1 : 0;
-    L->ws_stride = kHeaderWords * 4 + L->state_bytes;
-    L->qcnt_off = L->state_bytes + (size_t)L->S * 8;
+    // workspace record of a replica: 16 header words, the saved shared-memory state, the queue ring
+    L->gq_off = kHeaderWords * 4 + L->state_bytes;
+    L->ws_stride = L->gq_off + (size_t)L->QC * 8;
+    // a warp's shared memory: saved state, staged arrivals, queue window (64 entries), per-class queue counts
+    L->qwin_off = L->state_bytes + (size_t)L->S * 8;
+    L->qcnt_off = L->qwin_off + 64 * 8;
     L->smem_per_warp = L->qcnt_off + (any_classflow ? align_up((size_t)c->n_classes * 4, 16) : 0);
     if (!any_classflow) L->qcnt_off = 0;
     // Optional trace staging (environment FCSIM_TRACE_BULK=1): 2 x 32 records of 8 bytes in shared memory,
@@ -255,21 +262,29 @@ typedef void (*step_kernel_t)(const Params);
 // The step kernel compiled for one policy, for a register allocation that lets 6 or 5 CTAs reside on an SM, and
 // for what is recorded per slot (0 nothing, 1 trace only, 2 decided at run time; Algorithm 1 and the MC benchmark
 // exist in the run-time form only).
-template <int kPol>
-static step_kernel_t step_kernel_for(bool six, int rec) {
-    if (kPol >= 4 || rec == 2) return six ? fcsim_step_kernel<kPol, 6, 2> : fcsim_step_kernel<kPol, 5, 2>;
+template <int kPol, int kCtas>
+static step_kernel_t step_kernel_for(int rec) {
+    if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2>;
     constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 and 5 uninstantiated
-    if (rec == 1) return six ? fcsim_step_kernel<kP, 6, 1> : fcsim_step_kernel<kP, 5, 1>;
-    return six ? fcsim_step_kernel<kP, 6, 0> : fcsim_step_kernel<kP, 5, 0>;
+    if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1>;
+    return fcsim_step_kernel<kP, kCtas, 0>;
 }
-static step_kernel_t pick_step_kernel(int policy, bool six, int rec) {
+template <int kPol>
+static step_kernel_t step_kernel_for(int ctas, int rec) {
+    switch (ctas) {
+        case 5: return step_kernel_for<kPol, 5>(rec);
+        case 6: return step_kernel_for<kPol, 6>(rec);
+        default: return step_kernel_for<kPol, 7>(rec);
+    }
+}
+static step_kernel_t pick_step_kernel(int policy, int ctas, int rec) {
     switch (policy) {
-        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(six, rec);
-        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(six, rec);
-        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(six, rec);
-        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(six, rec);
-        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(six, rec);
-        case FCSIM_POLICY_MC: return step_kernel_for<5>(six, rec);
+        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(ctas, rec);
+        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(ctas, rec);
+        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(ctas, rec);
+        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec);
+        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec);
+        case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec);
         default: return nullptr;
     }
 }
@@ -568,8 +583,8 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
                 tab = block;
                 block += tab_extra;
             }
-            for (int six = 0; six <= 1; ++six) {
-                step_kernel_t k = pick_step_kernel(pl.policy, six != 0, rec);
+            for (int ctas = 5; ctas <= 7; ++ctas) {
+                step_kernel_t k = pick_step_kernel(pl.policy, ctas, rec);
                 if (!k) return fail(FCSIM_EINVAL);
                 e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
                 if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
@@ -621,7 +636,8 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     Params& p = h->params;
     std::memset(&p, 0, sizeof(p));
     p.M = cfg->M; p.K = cfg->K; p.Qcap = cfg->Qcap; p.Acap = cfg->Acap;
-    p.RC = L.RC; p.S = L.S; p.Apad = L.Apad;
+    p.S = L.S; p.Apad = L.Apad;
+    p.qmask = L.QC - 1; p.gq_off = (uint32_t)L.gq_off; p.qwin_off = (uint32_t)L.qwin_off;
     p.key0 = (uint32_t)(cfg->seed & 0xffffffffu);
     p.key1 = (uint32_t)(cfg->seed >> 32);
     p.n_classes = cfg->n_classes; p.n_groups = cfg->n_groups; p.n_replicas = (int)L.R;

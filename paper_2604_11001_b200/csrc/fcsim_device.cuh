@@ -2,27 +2,32 @@
 // under Algorithm 2, Algorithm 1, or one of the baselines (greedy, chunked prefill, alpha-protection greedy,
 // MC benchmark).
 //
-// Data layout per replica (shared memory while a warp owns the replica, the same bytes in the
-// caller's workspace between launches):
-//   ring  [RC]   u64   waiting queue and active set in ONE ring: entries head .. head+nP-1 are the
-//                      active set in activation order, the next nQ entries are the FIFO queue.
-//                      Because activation is FIFO and eviction is LIFO back to the queue front
-//                      (Section 3.3), the concatenation is always sorted by arrival, so activation
-//                      and eviction only move the boundary; nothing is copied.
+// Data layout per replica:
+//   ring  [Acap] u64   the active set in activation order, a ring in shared memory while a warp owns the replica
+//                      (the same bytes in the caller's workspace between launches);
 //                      entry = l | o << 16 | t_arr << 32 | class << 56.
-//   state [Acap] u32   one word per active entry (its own ring, same order): for a request whose
-//                      prompt is in the cache the slot in which its last token is generated
-//                      (t_fin = activation slot + o - 1, so its output count is implied by the
-//                      slot number and "process all requests" costs nothing); for a request still
-//                      prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so far;
-//                      0 for a request that has completed but whose entry has not been squeezed
-//                      out yet (completed entries are removed lazily, many at a time).
+//   state [Acap] u32   one word per active entry (same ring index): for a request whose prompt is in the cache
+//                      the slot in which its last token is generated (t_fin = activation slot + o - 1, so its
+//                      output count is implied by the slot number and "process all requests" costs nothing);
+//                      for a request still prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so
+//                      far; 0 for a request that has completed but whose entry has not been squeezed out yet
+//                      (completed entries are removed lazily, many at a time).
+//   vproj [Acap] i32   only with MC groups: projected memory usage of the last slot of each active entry.
+//   queue [QC]   u64   the FIFO waiting queue, a ring in the replica's record in GLOBAL memory (QC a power of
+//                      two >= Qcap + Acap: evictions may push the queue past Qcap).  It is touched at its ends
+//                      only: arrivals are appended (plain stores, nobody waits for them), the head is read
+//                      through qwin, evicted requests are pushed back on the head (Section 3.3: LIFO eviction
+//                      to the queue front keeps "active set, then queue" sorted by arrival).  Keeping the queue
+//                      out of shared memory is what lets more warps reside on an SM.
+//   qwin  [64]   u64   shared-memory copy of the queue entries with sequence numbers [wseq, wseq + 64), slot =
+//                      sequence number & 63; the head is always inside, and the window is topped up from global
+//                      memory 32 entries at a time, long before they are needed.
 //                      Under Algorithm 1 a pick may leave the middle of the queue (first request of a
 //                      class); the entries ahead of it then shift by one place.
-//   vproj [Acap] i32   only with MC groups: projected memory usage of the last slot of each active entry.
 //   stage [S]    u64   arrivals generated ahead of time for the next batch of <= 32 slots.
 //   qcnt  [classes] u32  only with Algorithm-1 groups: waiting requests per class.
-// Only ring, state and vproj are saved between launches (plus 16 scalar words); the rest is rebuilt.
+// Only ring, state and vproj are saved between launches (plus 16 scalar words); the queue lives in global memory
+// and the rest is rebuilt.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -71,7 +76,9 @@ struct DevGroup {
 };
 
 struct Params {
-    int32_t M, K, Qcap, Acap, RC, S, Apad;  // RC, Apad: padded storage sizes of the two rings
+    int32_t M, K, Qcap, Acap, S, Apad;  // Apad: padded storage size of the active ring
+    uint32_t qmask;               // queue ring size - 1 (a power of two)
+    uint32_t gq_off;              // byte offset of the queue ring in a replica's workspace record
     uint32_t key0, key1;
     int32_t n_classes, n_groups, n_replicas;  // n_groups: entries of `groups`
     int32_t n_work;               // replicas this launch advances (those of the groups in `groups`)
@@ -81,6 +88,7 @@ struct Params {
     const uint4* gpool;           // guide records {k0, thresholds k0, k0+1, k0+2}, one per bucket of u
     const int32_t* bclass;        // per-class budgets b_k of the Algorithm-1 groups
     uint32_t qcnt_off;            // byte offset of the per-class queue counts in a warp's shared memory (0 = none)
+    uint32_t qwin_off;            // byte offset of the queue window in a warp's shared memory
     uint32_t tabcache_off;        // byte offset in the CTA's shared memory of a copy of `tables` (0 = none)
     uint32_t state_bytes;         // ring + state words (+ projection words): what is saved between launches
     int32_t has_v;                // 1 = a projection word per active entry follows the state words (MC benchmark)
@@ -238,7 +246,7 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
     }
     return dummy[threadIdx.x];
 }
-#define RING(i) checked_ref(ring, (i), RC, __LINE__, p.debug, r)
+#define RING(i) checked_ref(ring, (i), Acap, __LINE__, p.debug, r)
 #define STATE(i) checked_ref(state, (i), Acap, __LINE__, p.debug, r)
 #define STAGE(i) checked_ref(stage, (i), S, __LINE__, p.debug, r)
 #define TROW(i) checked_ref(trow, (i), p.n_rec, __LINE__, p.debug, r)
@@ -286,14 +294,15 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
     const int warp = threadIdx.x >> 5;
     unsigned char* my = smem_raw + (size_t)warp * p.smem_per_warp;
     uint64_t* ring = reinterpret_cast<uint64_t*>(my);
-    uint32_t* state = reinterpret_cast<uint32_t*>(my + (size_t)p.RC * 8);
+    uint32_t* state = reinterpret_cast<uint32_t*>(my + (size_t)p.Apad * 8);
     // MC benchmark: vproj[k] = memory usage projected for the last slot of active entry k (same ring as state)
     int* vproj = reinterpret_cast<int*>(state + p.Apad);
     const int state_bytes = (int)p.state_bytes;  // multiple of 16 (host guarantees)
     uint64_t* stage = reinterpret_cast<uint64_t*>(my + state_bytes);
     uint32_t* qcnt = reinterpret_cast<uint32_t*>(my + p.qcnt_off);  // waiting requests per class (Algorithm 1 only)
+    uint64_t* qwin = reinterpret_cast<uint64_t*>(my + p.qwin_off);   // window on the queue head (64 entries)
 
-    const int RC = p.RC, Acap = p.Acap, Qcap = p.Qcap, M = p.M, K = p.K, S = p.S;
+    const int Acap = p.Acap, Qcap = p.Qcap, M = p.M, K = p.K, S = p.S;
     const bool kinf = (K == 0);
     const uint32_t FULL = 0xffffffffu;
     const uint32_t gt_mask = lanemask_gt();
@@ -333,8 +342,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         unsigned char* ws = p.workspace + (size_t)r * p.ws_stride;
         uint32_t* hdr = reinterpret_cast<uint32_t*>(ws);
         const uint32_t hw = (lane < kHeaderWords) ? hdr[lane] : 0u;
-        int head = (int)__shfl_sync(FULL, hw, 0);     // ring position of the oldest active entry
-        int shead = (int)__shfl_sync(FULL, hw, 1);    // same for the state ring
+        uint32_t qh = __shfl_sync(FULL, hw, 0);       // sequence number of the queue head (ring place = qh & qmask)
+        int shead = (int)__shfl_sync(FULL, hw, 1);    // ring position of the oldest active entry
         int nP = (int)__shfl_sync(FULL, hw, 2);       // entries in the active range, completed ones included
         int nQ = (int)__shfl_sync(FULL, hw, 3);
         int U = (int)__shfl_sync(FULL, hw, 4);        // usage carried out of the last slot, completions released
@@ -350,6 +359,42 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             uint4* dst = reinterpret_cast<uint4*>(my);
             for (int i = lane; i < state_bytes / 16; i += 32) dst[i] = src[i];
         }
+        // ---- the queue: ring in global memory, its head seen through the shared-memory window
+        uint64_t* __restrict__ gq = reinterpret_cast<uint64_t*>(ws + p.gq_off);
+        const uint32_t qmask = p.qmask;
+        uint32_t wseq = qh;  // the window holds the entries with sequence numbers [wseq, wseq + 64)
+        auto q_get = [&](uint32_t seq) -> uint64_t {  // seq in [qh, qh + nQ)
+            return (seq - wseq < 64u) ? qwin[seq & 63u] : gq[seq & qmask];
+        };
+        auto q_put = [&](uint32_t seq, uint64_t e) {  // global memory is always written, the window when it covers seq
+            gq[seq & qmask] = e;
+            if (seq - wseq < 64u) qwin[seq & 63u] = e;
+        };
+        // (re)load the part of the window from sequence number `from` on (all earlier queue writes of this warp
+        // must be behind a __syncwarp)
+        auto q_fill = [&](uint32_t from) {
+            for (uint32_t sq = from + (uint32_t)lane; sq - wseq < 64u; sq += 32u)
+                if (sq - qh < (uint32_t)nQ) qwin[sq & 63u] = gq[sq & qmask];
+            __syncwarp();
+        };
+        // one entry leaves at the head; when half of the window is used up it moves on by 32 entries
+        auto q_pop = [&]() {
+            ++qh;
+            --nQ;
+            if (qh - wseq >= 32u) {
+                wseq += 32u;
+                __syncwarp();
+                q_fill(wseq + 32u);
+            }
+        };
+        // an evicted request becomes the head again (lane 0 writes; callers synchronise the warp afterwards)
+        auto q_push_front = [&](uint64_t e) {
+            --qh;
+            ++nQ;
+            if ((int)(qh - wseq) < 0) wseq = qh;  // the window slides down by one; its last entry stays in global memory
+            if (lane == 0) q_put(qh, e);
+        };
+        q_fill(wseq);
         long long* cptr = p.counters + (size_t)r * C_COUNT;
         long long cnt = (lane < C_COUNT) ? cptr[lane] : 0;  // lane k owns counter k
         __syncwarp();
@@ -358,7 +403,6 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 #define CADD(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt += v__; } while (0)
 #define CMAX(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt = (cnt > v__) ? cnt : v__; } while (0)
 #define CSET(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt = v__; } while (0)
-#define WR(x) ((x) >= RC ? (x) - RC : (x))
 #define WA(x) ((x) >= Acap ? (x) - Acap : (x))
 
         // per-launch partial sums of the quantities touched every slot
@@ -414,18 +458,17 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 const int sh = holes + __popc(m & gt_mask);  // completed entries after this one
                 const bool mv = valid && !dead && sh > 0;
                 int v = 0;
-                if (mv) e = RING(WR(head + i));
+                if (mv) e = RING(WA(shead + i));
                 if (kExt && p.has_v && mv) v = vproj[WA(shead + i)];
                 __syncwarp();
                 if (mv) {
-                    RING(WR(head + i + sh)) = e;
+                    RING(WA(shead + i + sh)) = e;
                     STATE(WA(shead + i + sh)) = sw;
                     if (kExt && p.has_v) vproj[WA(shead + i + sh)] = v;
                 }
                 __syncwarp();
                 holes += __popc(m);
             }
-            head = WR(head + nD);
             shead = WA(shead + nD);
             nP -= nD;
             pf_lo = max(0, pf_lo - nD);
@@ -446,7 +489,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         if ((kExt && policy == 4)) {  // Algorithm 1 picks per class: count the waiting requests of every class
             for (int c = lane; c < p.n_classes; c += 32) qcnt[c] = 0;
             __syncwarp();
-            for (int i = lane; i < nQ; i += 32) atomicAdd(&qcnt[entry_cls(RING(WR(head + nP + i)))], 1u);
+            for (int i = lane; i < nQ; i += 32) atomicAdd(&qcnt[entry_cls(q_get(qh + (uint32_t)i))], 1u);
             __syncwarp();
         }
 
@@ -523,10 +566,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     const uint32_t info = __shfl_sync(FULL, packed, k);
                     const int sp = (int)(info >> 8);  // where the slot's arrivals are staged
                     const int acc = min((int)(info & 0xffu), Qcap - nQ);
-                    const int tail = WR(head + nP + nQ);
+                    const uint32_t tail = qh + (uint32_t)nQ;
                     for (int i = lane; i < acc; i += 32) {
                         const uint64_t e = STAGE(sp + i);
-                        RING(WR(tail + i)) = e;
+                        q_put(tail + (uint32_t)i, e);
                         if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
                     }
                     nQ += acc;
@@ -547,7 +590,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         uint64_t e = 0;
                         if (i < nP) sw = STATE(WA(shead + i));
                         const bool pf = (sw & kPrefillBit) != 0;
-                        if (pf) e = RING(WR(head + i));
+                        if (pf) e = RING(WA(shead + i));
                         const int pcur = (int)(sw & ~kPrefillBit);
                         const int l = entry_l(e);
                         const int d = pf ? min(chunk, l - pcur) : 0;
@@ -608,12 +651,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             const int b_k = __ldg(bk + kc);
                             for (int ak = 0; ak < b_k && qcnt[kc] > 0; ++ak) {
                                 if (nP == Acap) { storage_hit = true; break; }  // completed entries were squeezed out above
-                                const int q0 = head + nP;
+                                const uint32_t q0 = qh;
                                 int pos = -1;
                                 uint64_t e = 0;
                                 for (int base = 0; base < nQ && pos < 0; base += 32) {
                                     const int i = base + lane;
-                                    const uint64_t c = (i < nQ) ? RING(WR(q0 + i)) : 0;
+                                    const uint64_t c = (i < nQ) ? q_get(q0 + (uint32_t)i) : 0;
                                     const uint32_t m = __ballot_sync(FULL, i < nQ && entry_cls(c) == kc);
                                     if (m) {
                                         const int src = __ffs(m) - 1;
@@ -629,14 +672,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     const int i = base + lane;
                                     const bool mv = i < pos;
                                     uint64_t c = 0;
-                                    if (mv) c = RING(WR(q0 + i));
+                                    if (mv) c = q_get(q0 + (uint32_t)i);
                                     __syncwarp();
-                                    if (mv) RING(WR(q0 + i + 1)) = c;
+                                    if (mv) q_put(q0 + (uint32_t)i + 1u, c);
                                     __syncwarp();
                                 }
                                 const uint32_t sw = (uint32_t)(t + entry_o(e) - 1);
                                 if (lane == 0) {
-                                    RING(WR(q0)) = e;
+                                    RING(WA(shead + nP)) = e;
                                     STATE(WA(shead + nP)) = sw;
                                     qcnt[kc] -= 1;
                                 }
@@ -644,7 +687,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 if (lane == (nP >> bsh)) cmin = min(cmin, sw);
                                 Ndec++;
                                 nP++;
-                                nQ--;
+                                q_pop();  // the entries ahead of the pick moved up: the freed place is the head's
                                 G += l + 1;
                                 if (!kinf) R -= min(l, R);
                                 a++;
@@ -663,7 +706,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room
                             CADD(C_ACAP_BLOCKED, 1); status |= 1u; break;
                         }
-                        if (q_e == 0) q_e = RING(WR(head + nP));
+                        if (q_e == 0) q_e = qwin[qh & 63u];  // the head is always inside the window
                         const int l = entry_l(q_e);
                         int g, need;
                         if (policy == 2) {
@@ -707,7 +750,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 const bool in = i < nP;
                                 const int si = WA(shead + (in ? i : 0));
                                 const uint32_t swi = STATE(si);
-                                const uint64_t ei = RING(WR(head + (in ? i : 0)));
+                                const uint64_t ei = RING(WA(shead + (in ? i : 0)));
                                 const uint32_t vi = (uint32_t)vproj[si];
                                 const bool live = in && swi != kDead;
                                 uint32_t f_i = swi;
@@ -734,7 +777,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     if (swi != kDead) {
                                         int f_i = (int)swi;
                                         if (worst) {
-                                            const uint64_t ei = RING(WR(head + i));
+                                            const uint64_t ei = RING(WA(shead + i));
                                             f_i += tabs[1 + p.n_classes + entry_cls(ei)].vmin +
                                                    (int)tabs[1 + p.n_classes + entry_cls(ei)].n - 1 - entry_o(ei);
                                         }
@@ -757,10 +800,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             if (n_pref == 0) pf_lo = nP;
                             n_pref++;
                         }
-                        if (lane == 0) STATE(WA(shead + nP)) = sw;
+                        if (lane == 0) {
+                            RING(WA(shead + nP)) = q_e;
+                            STATE(WA(shead + nP)) = sw;
+                        }
                         __syncwarp();  // the next pick may scan the active range (MC projection) or squeeze it
                         nP++;
-                        nQ--;
+                        q_pop();
                         q_e = 0;
                         G += need;
                         if (!kinf) R -= min(g, R);
@@ -781,23 +827,26 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     int nev = 0, wasted = 0;
                     if (policy == 3) {
                         // alpha-protection greedy (Section 4.1): every active request goes back to the queue.
-                        // Completed entries were squeezed out above, so the whole active range is live and
-                        // simply becomes the front of the queue.
+                        // Completed entries were squeezed out above, so the whole active range is live and is
+                        // copied, in order, in front of the queue head.
                         long long kept_w = 0;
+                        const uint32_t nqh = qh - (uint32_t)nP;
+                        wseq = nqh;  // the window restarts at the new head (reloaded below)
                         for (int base = 0; base < nP; base += 32) {
                             const int i = base + lane;
                             if (i < nP) {
                                 const uint32_t sw = STATE(WA(shead + i));
+                                uint64_t e = RING(WA(shead + i));
                                 if (!(sw & kPrefillBit)) {
-                                    const uint64_t e = RING(WR(head + i));
                                     const int j = t - (int)sw + entry_o(e) - 1;
                                     wasted += j;
-                                    if (grp.keep != 0 && j > 0) {  // each lane rewrites its own entries only
+                                    if (grp.keep != 0 && j > 0) {
                                         const int l = entry_l(e);
                                         kept_w += (long long)l * j + (long long)j * (j + 1) / 2;
-                                        RING(WR(head + i)) = pack_entry(l + j, entry_o(e) - j, entry_tarr(e), entry_cls(e));
+                                        e = pack_entry(l + j, entry_o(e) - j, entry_tarr(e), entry_cls(e));
                                     }
                                 }
+                                gq[(nqh + (uint32_t)i) & qmask] = e;
                             }
                         }
                         wasted = __reduce_add_sync(FULL, wasted);
@@ -807,8 +856,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             wasted = 0;
                         }
                         nev = nP;
+                        qh = nqh;
                         nQ += nP;
                         nP = 0;
+                        __syncwarp();
+                        q_fill(wseq);
                         Ndec = 0;
                         n_pref = 0;
                         G = 0;
@@ -832,15 +884,15 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             }
                             i = found;
                             sw = STATE(WA(shead + i));
-                            const uint64_t moved = RING(WR(head + i));
+                            const uint64_t moved = RING(WA(shead + i));
                             __syncwarp();
                             if (lane == 0) {
-                                RING(WR(head + nP - 1)) = moved;
+                                RING(WA(shead + nP - 1)) = moved;
                                 STATE(WA(shead + i)) = kDead;
                             }
                             __syncwarp();
                         }
-                        uint64_t e = RING(WR(head + nP - 1));
+                        uint64_t e = RING(WA(shead + nP - 1));
                         if (sw & kPrefillBit) {
                             G -= (int)(sw & ~kPrefillBit);
                             n_pref--;
@@ -857,14 +909,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 CADD(C_COMPLETED_TOKENS, j);
                                 CADD(C_SUM_W_COMPLETED, (long long)l * j + (long long)j * (j + 1) / 2);
                                 e = pack_entry(l + j, entry_o(e) - j, entry_tarr(e), entry_cls(e));
-                                __syncwarp();  // every lane has read the old entry
-                                if (lane == 0) RING(WR(head + nP - 1)) = e;
                             }
                         }
+                        q_push_front(e);
                         q_e = e;
                         if ((kExt && policy == 4) && lane == 0) qcnt[entry_cls(e)] += 1;
                         nP--;
-                        nQ++;
                         nev++;
                     }
                     if (pf_lo > nP) pf_lo = nP;
@@ -893,7 +943,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             const bool in = vi < nP;
                             const int si = WA(shead + (in ? vi : 0));
                             const uint32_t swv = STATE(si);
-                            const uint64_t ev = RING(WR(head + (in ? vi : 0)));
+                            const uint64_t ev = RING(WA(shead + (in ? vi : 0)));
                             const bool live = in && swv != kDead;
                             const DevTable dv = tabs[1 + p.n_classes + (live ? entry_cls(ev) : 0)];
                             // a completed entry takes no correction: later than any slot
@@ -921,7 +971,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             uint64_t e = 0;
                             if (m) {
                                 if (done) {
-                                    e = RING(WR(head + i));
+                                    e = RING(WA(shead + i));
                                     const int l = entry_l(e), o = entry_o(e);
                                     const int lat = t - entry_tarr(e) + 1;
                                     acc_lat += (unsigned)lat;
@@ -1023,16 +1073,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             __syncwarp();
         }
         long long age = 0, resj = 0;
-        for (int i = lane; i < nP + nQ; i += 32) {
-            const uint64_t e = RING(WR(head + i));
-            bool live = true;
-            if (i < nP) {
-                const uint32_t sw = STATE(WA(shead + i));
-                live = (sw != kDead);
-                if (live && !(sw & kPrefillBit)) resj += t_end - (int)sw + entry_o(e);
+        __syncwarp();  // the queue entries written during the last slots are read by other lanes below
+        for (int i = lane; i < nP; i += 32) {
+            const uint64_t e = RING(WA(shead + i));
+            const uint32_t sw = STATE(WA(shead + i));
+            if (sw != kDead) {
+                if (!(sw & kPrefillBit)) resj += t_end - (int)sw + entry_o(e);
+                age += t_end - entry_tarr(e) + 1;
             }
-            if (live) age += t_end - entry_tarr(e) + 1;
         }
+        for (int i = lane; i < nQ; i += 32) age += t_end - entry_tarr(gq[(qh + (uint32_t)i) & qmask]) + 1;
         age = warp_sum64(age);
         resj = warp_sum64(resj);
         CADD(C_SUM_U, sumU);
@@ -1059,7 +1109,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 
         uint32_t out = 0;
         switch (lane) {
-            case 0: out = (uint32_t)head; break;
+            case 0: out = qh; break;
             case 1: out = (uint32_t)shead; break;
             case 2: out = (uint32_t)nP; break;
             case 3: out = (uint32_t)nQ; break;
@@ -1084,7 +1134,6 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 #undef CADD
 #undef CMAX
 #undef CSET
-#undef WR
 #undef WA
     }
 }

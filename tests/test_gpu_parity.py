@@ -151,10 +151,10 @@ def test_trace_bulk_copy_variant(monkeypatch):
 
 
 def test_maximum_sizes():
-    # lengths at the 16-bit limit, capacity 2^30, rings so large that a CTA holds a single warp,
+    # lengths at the 16-bit limit, capacity 2^30, an active ring so large that a CTA holds a single warp,
     # 255 arrivals in a slot, the largest flow rate
     big = wl.SimConfig(
-        M=1 << 30, K=0, T_max=300, Qcap=9000, Acap=8000, seed=(1 << 63) + 5, class_law=wl.constant_table(0),
+        M=1 << 30, K=0, T_max=300, Qcap=9000, Acap=16000, seed=(1 << 63) + 5, class_law=wl.constant_table(0),
         prompt=(wl.uniform_table(65000, 65535),), decode=(wl.table_from_pmf(1, [0.5] + [0.0] * 65533 + [0.5]),),
         arrivals=(wl.Arrivals((wl.table_from_pmf(0, [0.5] + [0.0] * 254 + [0.5]),)),),
         groups=(wl.Group(wl.POLICY_FLOW, b_fp=0xFFFFFFFF, n_replicas=3),
@@ -197,7 +197,7 @@ def test_handles_with_different_shared_memory_needs_coexist():
     # a handle that needs more than the default 48 KB of shared memory per CTA must keep working after a
     # smaller one has been created (the opt-in limit belongs to the kernel, not to the handle)
     from paper_2604_11001_b200 import binding as fb
-    big_cfg = degenerate_config(n=20, l=1, o=3, policy="greedy", b=0, K=0, c=0, M=100000, T=60, Qcap=2000, Acap=1500)
+    big_cfg = degenerate_config(n=20, l=1, o=3, policy="greedy", b=0, K=0, c=0, M=100000, T=60, Qcap=2000, Acap=5000)
     big_cfg = big_cfg.with_(decode=(wl.uniform_table(1, 40),))
     small_cfg = wl.config1(replicas=4, T=60)
     big = fb.Simulation(big_cfg)
