@@ -158,7 +158,8 @@ typedef struct {
 } fcsim_summary;
 
 /* DEVICE buffers, caller-owned, each at least the size fcsim_query_sizes reports and 16-byte aligned.
- * workspace: per-replica simulator state between launches (scratch; opaque).
+ * workspace: per replica, the simulator state between launches and the waiting queue (a ring of the next power of
+ *            two >= Qcap + Acap entries of 8 bytes, read and written during launches); opaque.
  * counters:  [R] fcsim_counters.
  * trace:     [R][T_max / trace_stride] {int32 U_t, int32 |Q_t|}, or NULL when trace_stride = 0.
  * hist:      [R][hist_bins] int32, or NULL when hist_bins = 0.
