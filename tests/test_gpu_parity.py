@@ -302,3 +302,21 @@ def test_policies_interleaved_over_groups_on_a_side_stream():
         gpu[name] = None if v is None else v.cpu().numpy()
     sim.close()
     assert_same(cfg, gpu, ref, 1200, "interleaved policies")
+
+
+def test_dense_tables_take_the_guide_fall_back_search():
+    # length laws with far more thresholds than a guide has buckets (60 000 equiprobable prompt lengths: about four
+    # thresholds per bucket, so every fifth lookup must finish with the search behind the guide record), an arrival
+    # count law with mass at both ends, and a class law with a class of probability zero
+    prompt = (wl.uniform_table(1, 60000), wl.uniform_table(7, 7), wl.table_from_pmf(3, [0.999] + [1e-3 / 4999] * 4999))
+    decode = (wl.uniform_table(1, 300), wl.geometric_table(3.0, 4000), wl.uniform_table(2, 3))
+    cfg = wl.SimConfig(
+        M=4000000, K=0, T_max=500, Qcap=64, Acap=256, seed=77, class_law=wl.table_from_pmf(0, [0.6, 0.0, 0.4]),
+        prompt=prompt, decode=decode,
+        arrivals=(wl.Arrivals((wl.table_from_pmf(0, [0.55] + [0.0] * 2 + [0.4] + [0.0] * 26 + [0.05]),)),),
+        groups=(wl.Group(wl.POLICY_FLOW, b_fp=wl.b_to_fp(2.5), n_replicas=6),
+                wl.Group(wl.POLICY_GREEDY, n_replicas=6, rng_replica_base=100)),
+        trace_stride=1, hist_bins=32, hist_shift=5, complog_cap=4096)
+    ref = orc.run(cfg, threads=4)
+    assert ref["counters"][:, orc.CIDX["completed"]].min() > 200
+    assert_same(cfg, run_gpu(cfg, pieces=[123, 377]), ref, 500, "dense tables")
