@@ -443,8 +443,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
         int2* lrow = (kRec == 2 && p.complog) ? p.complog + (size_t)r * p.complog_cap : nullptr;
 
-        // Squeeze the completed entries out of the active range: survivors slide towards the queue
-        // boundary (right-to-left pass), the head advances, the queue is not touched.
+        // Squeeze the completed entries out of the active range: survivors slide towards the newest end
+        // (right-to-left pass) and the oldest end of the ring advances.
         auto compact = [&]() {
             int holes = 0;
             for (int base = (nP - 1) & ~31; base >= 0; base -= 32) {
@@ -873,8 +873,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         uint32_t sw = STATE(WA(shead + i));
                         if (sw == kDead) {
                             // completed entries lie on top of the newest live one: find it (backwards, 32 at a
-                            // time), and move it to the top place, next to the queue, where it becomes the
-                            // queue head; its old place joins the completed entries
+                            // time), and move it to the top place, from where it is evicted below; its old
+                            // place joins the completed entries
                             int found = -1;
                             for (int top = nP; found < 0 && top > 0; top -= 32) {
                                 const int idx = top - 32 + lane;
