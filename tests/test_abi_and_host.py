@@ -39,7 +39,9 @@ def test_query_sizes_of_the_presets():
     assert s["trace"] == 64 * 2000 * 8
     assert s["hist"] == 64 * 1024 * 4
     assert s["complog"] == 64 * 2048 * 8
-    assert s["workspace"] % 16 == 0 and s["workspace"] >= 64 * (128 + 256) * 8
+    # per replica: 16 header words, the active ring (Acap entries of 8 + 4 bytes), the queue ring (next power of two
+    # >= Qcap + Acap entries of 8 bytes)
+    assert s["workspace"] == 64 * (64 + 256 * 12 + 512 * 8)
     s5 = fb.fcsim_query_sizes(wl.config5())
     assert s5["trace"] == 0 and s5["complog"] == 0 and s5["hist"] == 262144 * 1024 * 4
 
