@@ -10,8 +10,9 @@
 //                      the slot in which its last token is generated (t_fin = activation slot + o - 1, so its
 //                      output count is implied by the slot number and "process all requests" costs nothing);
 //                      for a request still prefilling (chunked policy) 0x80000000 | prompt tokens prefilled so
-//                      far; 0 for a request that has completed but whose entry has not been squeezed out yet
-//                      (completed entries are removed lazily, many at a time).
+//                      far; 0x40000000 | slot of completion for a request that has completed but whose entry
+//                      has not been squeezed out yet (completed entries are removed lazily, many at a time,
+//                      and their latency statistics are taken then, one entry per lane).
 //   vproj [Acap] i32   only with MC groups: projected memory usage of the last slot of each active entry.
 //   queue [QC]   u64   the FIFO waiting queue, a ring in the replica's record in GLOBAL memory (QC a power of
 //                      two >= Qcap + Acap: evictions may push the queue past Qcap).  It is touched at its ends
@@ -38,7 +39,9 @@ constexpr int kWarpsPerBlock = 4;
 constexpr int kHeaderWords = 16;  // per-replica scalar state kept in the workspace
 constexpr uint32_t kNoFin = 0xFFFFFFFFu;
 constexpr uint32_t kPrefillBit = 0x80000000u;
-constexpr uint32_t kDead = 0u;        // state word of a completed entry awaiting removal
+constexpr uint32_t kDead = 0x40000000u;  // state word of a completed entry awaiting removal: kDead | slot of completion
+                                         // (its latency statistics are taken when it is squeezed out)
+__device__ __forceinline__ bool is_dead(uint32_t sw) { return (sw >> 30) == 1u; }  // bit 31 marks a prefilling entry
 
 enum CounterIdx {
     C_STEPS_DONE = 0, C_STATUS, C_ARRIVED, C_DROPPED, C_ADMITTED, C_COMPLETED, C_EVICTIONS,
@@ -453,12 +456,22 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 uint32_t sw = kDead;
                 uint64_t e = 0;
                 if (valid) sw = STATE(WA(shead + i));
-                const bool dead = valid && (sw == kDead);
+                const bool dead = valid && is_dead(sw);
                 const uint32_t m = __ballot_sync(FULL, dead);
                 const int sh = holes + __popc(m & gt_mask);  // completed entries after this one
                 const bool mv = valid && !dead && sh > 0;
                 int v = 0;
-                if (mv) e = RING(WA(shead + i));
+                if (mv || dead) e = RING(WA(shead + i));
+                if (dead) {
+                    // the statistics of the completions, 32 at a time instead of one lane at a time
+                    const int l = entry_l(e), o = entry_o(e);
+                    const int lat = (int)(sw & ~kDead) - entry_tarr(e) + 1;
+                    acc_lat += (unsigned)lat;
+                    acc_o += (unsigned)o;
+                    acc_maxlat = max(acc_maxlat, lat);
+                    acc_w += (unsigned long long)l * o + (unsigned long long)o * (o + 1) / 2;
+                    if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
+                }
                 if (kExt && p.has_v && mv) v = vproj[WA(shead + i)];
                 __syncwarp();
                 if (mv) {
@@ -480,7 +493,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             for (int base = 0; base < nP; base += 32) {
                 const int i = base + lane;
                 const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
-                const uint32_t m = __reduce_min_sync(FULL, sw == kDead ? kNoFin : sw);
+                const uint32_t m = __reduce_min_sync(FULL, is_dead(sw) ? kNoFin : sw);
                 if (lane == (base >> bsh)) cmin = min(cmin, m);
             }
             next_fin = __reduce_min_sync(FULL, cmin);
@@ -752,7 +765,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 const uint32_t swi = STATE(si);
                                 const uint64_t ei = RING(WA(shead + (in ? i : 0)));
                                 const uint32_t vi = (uint32_t)vproj[si];
-                                const bool live = in && swi != kDead;
+                                const bool live = in && !is_dead(swi);
                                 uint32_t f_i = swi;
                                 if (worst) {
                                     const DevTable d = tabs[1 + p.n_classes + (live ? entry_cls(ei) : 0)];
@@ -774,7 +787,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 for (int base = 0; base < nP; base += 32) {
                                     const int i = base + lane;
                                     const uint32_t swi = (i < nP) ? STATE(WA(shead + i)) : kDead;
-                                    if (swi != kDead) {
+                                    if (!is_dead(swi)) {
                                         int f_i = (int)swi;
                                         if (worst) {
                                             const uint64_t ei = RING(WA(shead + i));
@@ -871,24 +884,27 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     while (policy != 3 && G > M && nP > nD) {
                         int i = nP - 1;
                         uint32_t sw = STATE(WA(shead + i));
-                        if (sw == kDead) {
+                        if (is_dead(sw)) {
                             // completed entries lie on top of the newest live one: find it (backwards, 32 at a
-                            // time), and move it to the top place, from where it is evicted below; its old
-                            // place joins the completed entries
+                            // time), and let it change places with the completed entry at the top (whose record
+                            // is still needed for its statistics); it is evicted from the top place below
+                            const uint32_t sw_top = sw;
                             int found = -1;
                             for (int top = nP; found < 0 && top > 0; top -= 32) {
                                 const int idx = top - 32 + lane;
                                 const uint32_t w = (idx >= 0) ? STATE(WA(shead + idx)) : kDead;
-                                const uint32_t m = __ballot_sync(FULL, w != kDead);
+                                const uint32_t m = __ballot_sync(FULL, !is_dead(w));
                                 if (m) found = top - 1 - __clz(m);
                             }
                             i = found;
                             sw = STATE(WA(shead + i));
                             const uint64_t moved = RING(WA(shead + i));
+                            const uint64_t top_e = RING(WA(shead + nP - 1));
                             __syncwarp();
                             if (lane == 0) {
                                 RING(WA(shead + nP - 1)) = moved;
-                                STATE(WA(shead + i)) = kDead;
+                                RING(WA(shead + i)) = top_e;
+                                STATE(WA(shead + i)) = sw_top;
                             }
                             __syncwarp();
                         }
@@ -944,7 +960,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             const int si = WA(shead + (in ? vi : 0));
                             const uint32_t swv = STATE(si);
                             const uint64_t ev = RING(WA(shead + (in ? vi : 0)));
-                            const bool live = in && swv != kDead;
+                            const bool live = in && !is_dead(swv);
                             const DevTable dv = tabs[1 + p.n_classes + (live ? entry_cls(ev) : 0)];
                             // a completed entry takes no correction: later than any slot
                             const int f_v = live ? (int)swv + dv.vmin + (int)dv.n - 1 - entry_o(ev) : 0x3fffffff;
@@ -972,19 +988,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             if (m) {
                                 if (done) {
                                     e = RING(WA(shead + i));
-                                    const int l = entry_l(e), o = entry_o(e);
-                                    const int lat = t - entry_tarr(e) + 1;
-                                    acc_lat += (unsigned)lat;
-                                    acc_o += (unsigned)o;
-                                    sum_lo += l + o;
-                                    acc_maxlat = max(acc_maxlat, lat);
-                                    acc_w += (unsigned long long)l * o + (unsigned long long)o * (o + 1) / 2;
-                                    if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
+                                    sum_lo += entry_l(e) + entry_o(e);
                                     if (lrow) {
                                         const int li = n_logged + ndone + __popc(m & lt_mask);  // activation order
-                                        if (li < p.complog_cap) LROW(li) = make_int2(t, lat);
+                                        if (li < p.complog_cap) LROW(li) = make_int2(t, t - entry_tarr(e) + 1);
                                     }
-                                    STATE(WA(shead + i)) = kDead;
+                                    // latency, workload and histogram of the completion are taken when the entry
+                                    // is squeezed out, many entries at a time
+                                    STATE(WA(shead + i)) = kDead | (uint32_t)t;
                                 }
                                 ndone += __popc(m);
                                 if (kExt && policy == 5 && grp.mc_worst != 0) {
@@ -1006,7 +1017,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     npend += cntm;
                                 }
                             }
-                            gmin = min(gmin, __reduce_min_sync(FULL, (done || sw == kDead) ? kNoFin : sw));
+                            gmin = min(gmin, __reduce_min_sync(FULL, (done || is_dead(sw)) ? kNoFin : sw));
                         }
                         if (lane == c) cmin = gmin;
                     }
@@ -1072,12 +1083,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             if (lane == 0) bulk_wait_all();
             __syncwarp();
         }
+        if (nD > 0) {  // the completions still inside the active range are accounted for before the replica is put back
+            __syncwarp();
+            compact();
+        }
         long long age = 0, resj = 0;
         __syncwarp();  // the queue entries written during the last slots are read by other lanes below
         for (int i = lane; i < nP; i += 32) {
             const uint64_t e = RING(WA(shead + i));
             const uint32_t sw = STATE(WA(shead + i));
-            if (sw != kDead) {
+            if (!is_dead(sw)) {
                 if (!(sw & kPrefillBit)) resj += t_end - (int)sw + entry_o(e);
                 age += t_end - entry_tarr(e) + 1;
             }
