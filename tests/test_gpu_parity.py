@@ -320,3 +320,14 @@ def test_dense_tables_take_the_guide_fall_back_search():
     ref = orc.run(cfg, threads=4)
     assert ref["counters"][:, orc.CIDX["completed"]].min() > 200
     assert_same(cfg, run_gpu(cfg, pieces=[123, 377]), ref, 500, "dense tables")
+
+
+def test_index_checked_build_records_no_violation():
+    # the same kernels compiled with every shared-memory and output index compared with its bound, over random
+    # configurations of all policies and cuts of the presets; run in a process of its own (one build per process)
+    import subprocess
+    import sys
+    runner = os.path.join(os.path.dirname(os.path.abspath(__file__)), "checked_runner.py")
+    out = subprocess.run([sys.executable, runner], capture_output=True, text=True, timeout=1500)
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "violations: 0" in out.stdout, out.stdout[-2000:]
