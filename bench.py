@@ -261,7 +261,7 @@ def main():
     # end to end through the host-buffer entry point: tables from host memory, every output back to host
     e2e = None
     out_bytes = sizes["counters"] + sizes["trace"] + sizes["hist"] + sizes["complog"]
-    if not args.no_e2e and out_bytes > 8e9:
+    if not args.no_e2e and out_bytes > 16e9:
         e2e = {"value": None, "unit": UNIT,
                "skipped": "outputs of %.1f GB are not copied to host buffers in the default run" % (out_bytes / 1e9)}
     elif not args.no_e2e:
