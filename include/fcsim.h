@@ -20,7 +20,7 @@
  * and owned by the caller; the library only allocates small private device copies of the tables.
  * One GPU; a handle is bound to the device that is current in fcsim_create, and fcsim_run / fcsim_stats
  * return FCSIM_EINVAL when called with another device current.  A handle is not thread-safe: calls on the
- * same handle must not overlap.
+ * same handle must not overlap.  Different handles may be driven from different threads.
  */
 #ifndef FCSIM_H
 #define FCSIM_H

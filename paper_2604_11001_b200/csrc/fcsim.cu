@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -258,6 +259,11 @@ void launch_reduce_hist(const int* hist, const DevGroup* groups, int G, int R, i
 }  // namespace
 
 typedef void (*step_kernel_t)(const Params);
+
+// The opt-in shared-memory limit is a property of a kernel, shared by every handle of the process: setting it
+// and using it (occupancy query, launch) happen under this lock, so that handles driven from different threads do
+// not change it between another handle's two steps.
+static std::mutex g_kernel_attr_mutex;
 
 // The step kernel compiled for one policy, for a register allocation that lets 6 or 5 CTAs reside on an SM, and
 // for what is recorded per slot (0 nothing, 1 trace only, 2 decided at run time; Algorithm 1 and the MC benchmark
@@ -586,10 +592,12 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
             for (int ctas = 5; ctas <= 7; ++ctas) {
                 step_kernel_t k = pick_step_kernel(pl.policy, ctas, rec);
                 if (!k) return fail(FCSIM_EINVAL);
-                e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
-                if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
                 int occ = 0;
-                e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, w * 32, block);
+                {
+                    std::lock_guard<std::mutex> lock(g_kernel_attr_mutex);
+                    e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
+                    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, w * 32, block);
+                }
                 if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
                 if (occ * w > best_warps) {
                     best_warps = occ * w;
@@ -692,10 +700,13 @@ extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
             p.n_work = pl.n_work;
             p.work_counter = h->d_work + pl.policy;
             p.tabcache_off = (uint32_t)pl.tabcache_off;
-            // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
-            CUDA_TRY(h, cudaFuncSetAttribute(pl.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_block));
-            pl.kernel<<<pl.grid, pl.warps_per_block * 32, pl.smem_block, ls>>>(p);
-            CUDA_TRY(h, cudaGetLastError());
+            {
+                // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
+                std::lock_guard<std::mutex> lock(g_kernel_attr_mutex);
+                CUDA_TRY(h, cudaFuncSetAttribute(pl.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_block));
+                pl.kernel<<<pl.grid, pl.warps_per_block * 32, pl.smem_block, ls>>>(p);
+                CUDA_TRY(h, cudaGetLastError());
+            }
             if (pl.side) CUDA_TRY(h, cudaEventRecord(pl.done, pl.side));
         }
         for (const PolicyLaunch& pl : h->launches)

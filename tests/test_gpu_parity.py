@@ -331,3 +331,36 @@ def test_index_checked_build_records_no_violation():
     out = subprocess.run([sys.executable, runner], capture_output=True, text=True, timeout=1500)
     assert out.returncode == 0, out.stderr[-2000:]
     assert "violations: 0" in out.stdout, out.stdout[-2000:]
+
+
+def test_two_handles_driven_from_two_threads():
+    # handles with different shared-memory needs use the same kernels; each thread creates its handle, runs it in
+    # many short calls and reads its statistics while the other does the same
+    import threading
+    from paper_2604_11001_b200 import binding as fb
+    big_cfg = degenerate_config(n=20, l=1, o=3, policy="greedy", b=0, K=0, c=0, M=100000, T=400, Qcap=2000, Acap=5000)
+    big_cfg = big_cfg.with_(decode=(wl.uniform_table(1, 40),))
+    small_cfg = wl.config1(replicas=8, T=400)
+    out, errors = {}, []
+
+    def drive(name, cfg):
+        try:
+            import torch
+            stream = torch.cuda.Stream()
+            sim = fb.Simulation(cfg)
+            for _ in range(40):
+                sim.run(10, stream)
+            out[name] = sim.stats(stream)[0]
+            sim.close()
+        except Exception as e:   # reported by the main thread
+            errors.append((name, repr(e)))
+
+    threads = [threading.Thread(target=drive, args=("big", big_cfg)),
+               threading.Thread(target=drive, args=("small", small_cfg))]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors
+    assert (out["big"] == orc.run(big_cfg)["counters"]).all()
+    assert (out["small"] == orc.run(small_cfg)["counters"]).all()
