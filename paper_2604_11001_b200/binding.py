@@ -88,7 +88,7 @@ def load():
     if os.environ.get("FCSIM_LIB"):           # explicit library path (diagnostic builds)
         path = os.environ["FCSIM_LIB"]
     elif os.environ.get("FCSIM_CHECKED"):     # index-checked diagnostic build
-        path = _build.LIB_CHECKED if os.path.exists(_build.LIB_CHECKED) else _build.build(checked=True)
+        path = _build.build(checked=True)      # compiled if missing or older than the sources
     else:
         path = _build.LIB
         if not os.path.exists(path) or os.environ.get("FCSIM_REBUILD"):

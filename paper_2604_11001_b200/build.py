@@ -13,10 +13,10 @@ SOURCES = [os.path.join(CSRC, "fcsim.cu")]
 HEADERS = [os.path.join(CSRC, "fcsim_device.cuh"), os.path.join(ROOT, "include", "fcsim.h")]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(f) > t for f in SOURCES + HEADERS)
 
 
@@ -27,6 +27,8 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
     """Compile if the sources are newer than the library; returns the library path.
     ``checked`` builds the index-checked diagnostic variant (libfcsim_checked.so)."""
     if checked:
+        if not force and not _stale(LIB_CHECKED):
+            return LIB_CHECKED
         return _compile(LIB_CHECKED, verbose, ["-DFCSIM_CHECKED"])
     if not force and not _stale():
         return LIB
