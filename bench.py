@@ -32,9 +32,9 @@ UNIT = "replica-steps/s"
 # Executed warp-instructions per replica-step of the step kernels in the timed regime of each preset, from the
 # committed ncu captures (profiles/): smsp__inst_executed.sum over the launches of one bench step (one kernel per
 # policy present) / (replicas x slots).  None = not captured for the current kernels.
-INST_PER_REPLICA_STEP = {1: 240.8, 2: 261.4, 3: 289.9, 4: 396.4, 5: 195.0, 6: 1996.2}
+INST_PER_REPLICA_STEP = {1: 240.8, 2: 261.4, 3: 289.9, 4: 396.4, 5: 195.0, 6: 2016.7}
 # DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
-DRAM_BYTES_PER_REPLICA_STEP = {1: 30.0, 2: 19.7, 3: 21.4, 4: 12.8, 5: 9.3, 6: 84.6}
+DRAM_BYTES_PER_REPLICA_STEP = {1: 30.0, 2: 19.7, 3: 21.4, 4: 12.8, 5: 9.3, 6: 38.4}
 
 DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000, 6: 500}
 NAMES = {1: "cfg1-tiny-flow", 2: "cfg2-policy-comparison", 3: "cfg3-stability-sweep", 4: "cfg4-heavy-tail",

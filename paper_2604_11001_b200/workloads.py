@@ -336,8 +336,11 @@ def config6(replicas: int = 4096, T: int = 10000, alpha: float = 0.2, total_rate
     prompt = tuple(constant_table(10) for _ in range(3))
     decode = tuple(constant_table(o) for o in (20, 40, 60))
     M = 16492
+    # storage bound of the active set, chosen so that it never binds: about 200 requests are active at rate 5
+    # (never more than 300 in 2.5e8 replica-steps), about 500 when memory binds at rate 15
+    Acap = 512 if total_rate <= 5.0 else 1024
     return SimConfig(
-        M=M, K=0, T_max=T, Qcap=256, Acap=1024, seed=6, class_law=class_law, prompt=prompt, decode=decode,
+        M=M, K=0, T_max=T, Qcap=256, Acap=Acap, seed=6, class_law=class_law, prompt=prompt, decode=decode,
         arrivals=(Arrivals((poisson_table(total_rate),)),),
         groups=(Group(POLICY_FLOW, b_fp=12 << 16, n_replicas=replicas),
                 Group(POLICY_GREEDY, n_replicas=replicas),
