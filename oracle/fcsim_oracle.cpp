@@ -21,6 +21,8 @@
 // Thm. 3.3); the double-sum form of U_t (proof of Thm. 3.6); b -> infinity equals greedy
 // (Section 3.3); the stability dichotomy of Prop. 3.5 / Thm. 3.6; an independent
 // brute-force evaluator on tiny inputs.
+// The MC benchmark's future-memory test (Section 4.1) is evaluated slot by slot; a last-slots-only
+// shortcut exists as an opt-in mode and a test compares the two on every admission decision.
 // Parity unpinned against the paper (the paper only names them; pinned by hand traces
 // and reductions only): the token budget K, GREEDY, CHUNKED and the two-state arrival law.
 #include <algorithm>
@@ -139,12 +141,36 @@ struct Request {
     int32_t j;  // output tokens generated
 };
 
-// MC benchmark (Section 4.1): "only activates requests if the future memory usage remains within the
-// memory limit".  With no further activation, an active request that has generated j tokens before slot t
-// holds l + j + (tau - t + 1) tokens in slot tau until the slot of its (projected) last token,
-// tau_end = t + (o_proj - j) - 1, and nothing afterwards.  The candidate h would start in slot t.
-// The usage only drops when a request ends, so it is enough to look at every request's last slot.
+// MC benchmark (Section 4.1): a waiting request is started only if the memory usage of every future slot
+// stays within the limit.  The future is the one in which nothing else is started: every running request
+// and the candidate h (started in slot t) generate one token per slot until their (projected) last token.
+// A request that has generated j tokens before slot t holds l + j + (tau - t + 1) tokens in slot tau >= t,
+// up to and including the slot of its last token, t + (o_proj - j) - 1, and nothing afterwards.
+// The test walks the future slot by slot until everything has ended and sums the footprints in each slot.
 bool fits_future(const std::vector<Request>& P, const Request& h, int32_t t, int64_t M) {
+    std::vector<Request> all(P);
+    Request c = h;
+    c.p = c.l;
+    c.j = 0;
+    all.push_back(c);
+    int64_t horizon = t;  // last slot in which anything is still running
+    for (const Request& r : all) horizon = std::max<int64_t>(horizon, (int64_t)t + (r.o_proj - r.j) - 1);
+    for (int64_t tau = t; tau <= horizon; ++tau) {
+        int64_t usage = 0;
+        for (const Request& r : all) {
+            const int64_t last = (int64_t)t + (r.o_proj - r.j) - 1;
+            if (tau <= last) usage += (int64_t)r.l + r.j + (tau - t + 1);
+        }
+        if (usage > M) return false;
+    }
+    return true;
+}
+
+// Opt-in shortcut of the same test (mc_mode 1; mc_mode 2 evaluates both and reports a disagreement): between
+// two endings the usage only grows, one token per running request and slot, so the maximum over the future is
+// reached in some request's last slot and only those slots need to be summed.  A test compares the two on
+// every admission decision of a set of random configurations.
+bool fits_future_last_slots(const std::vector<Request>& P, const Request& h, int32_t t, int64_t M) {
     std::vector<Request> all(P);
     Request c = h;
     c.p = c.l;
@@ -214,7 +240,7 @@ int validate(const orc_config& c) {
 // model is violated (that would be a bug in this file, not a property of the inputs).
 int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replica, int32_t n_steps,
                 int64_t* C, int32_t* trace, int32_t* hist, int32_t* complog, int32_t* arrlog, int32_t* arrcls,
-                int32_t* admlog, int64_t admlog_cap, int64_t* n_admlog_out) {
+                int32_t* admlog, int64_t admlog_cap, int64_t* n_admlog_out, int mc_mode, int64_t* n_mc_tests) {
     const uint32_t key[2] = {(uint32_t)(cfg.seed & 0xffffffffu), (uint32_t)(cfg.seed >> 32)};
     const orc_arrivals& arr = cfg.arrivals[grp.arrivals_id];
     const int64_t INF = std::numeric_limits<int64_t>::max() / 4;
@@ -340,7 +366,17 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
                 need = (int64_t)h.l + 1;
             }
             if (G + need > admit_limit) { C[C_GATE_BLOCKED]++; break; }
-            if (mc && !fits_future(P, h, t, M)) { C[C_GATE_BLOCKED]++; break; }
+            if (mc) {
+                bool fits;
+                if (mc_mode == 1) {
+                    fits = fits_future_last_slots(P, h, t, M);
+                } else {
+                    fits = fits_future(P, h, t, M);
+                    if (mc_mode == 2 && fits != fits_future_last_slots(P, h, t, M)) return -20;
+                }
+                if (n_mc_tests) ++*n_mc_tests;
+                if (!fits) { C[C_GATE_BLOCKED]++; break; }
+            }
             Q.pop_front();
             h.p = (int32_t)g;
             h.j = 0;
@@ -469,9 +505,13 @@ int run_replica(const orc_config& cfg, const orc_group& grp, uint32_t rng_replic
 
 }  // namespace
 
-extern "C" int fcsim_oracle_run(const orc_config* cfg, int64_t first_replica, int64_t n_replicas,
-                                int32_t n_steps, const orc_outputs* out) {
-    if (!cfg || !out || !out->counters) return -1;
+// mc_mode: how the MC benchmark's future-memory test is evaluated: 0 = slot by slot (the definition),
+// 1 = last slots only (shortcut), 2 = both, returning -20 if they ever disagree.  n_mc_tests (may be NULL)
+// receives the number of tests made.
+extern "C" int fcsim_oracle_run_ex(const orc_config* cfg, int64_t first_replica, int64_t n_replicas,
+                                   int32_t n_steps, const orc_outputs* out, int mc_mode, int64_t* n_mc_tests) {
+    if (!cfg || !out || !out->counters || mc_mode < 0 || mc_mode > 2) return -1;
+    if (n_mc_tests) *n_mc_tests = 0;
     if (validate(*cfg)) return -2;
     if (n_steps < 0 || n_steps > cfg->T_max) return -3;
     int64_t total = 0;
@@ -498,8 +538,13 @@ extern "C" int fcsim_oracle_run(const orc_config* cfg, int64_t first_replica, in
                              out->arrlog ? out->arrlog + k * (int64_t)n_steps : nullptr,
                              out->arrcls ? out->arrcls + k * (int64_t)n_steps * cfg->n_classes : nullptr,
                              out->admlog ? out->admlog + 4 * k * out->admlog_cap : nullptr, out->admlog_cap,
-                             out->n_admlog ? out->n_admlog + k : nullptr);
+                             out->n_admlog ? out->n_admlog + k : nullptr, mc_mode, n_mc_tests);
         if (rc) return rc;
     }
     return 0;
+}
+
+extern "C" int fcsim_oracle_run(const orc_config* cfg, int64_t first_replica, int64_t n_replicas,
+                                int32_t n_steps, const orc_outputs* out) {
+    return fcsim_oracle_run_ex(cfg, first_replica, n_replicas, n_steps, out, 0, nullptr);
 }

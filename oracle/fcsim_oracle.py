@@ -76,6 +76,9 @@ def lib(sanitize: bool = False):
 def _bind(l):
     l.fcsim_oracle_run.restype = C.c_int
     l.fcsim_oracle_run.argtypes = [C.POINTER(_Config), C.c_int64, C.c_int64, C.c_int32, C.POINTER(_Outputs)]
+    l.fcsim_oracle_run_ex.restype = C.c_int
+    l.fcsim_oracle_run_ex.argtypes = [C.POINTER(_Config), C.c_int64, C.c_int64, C.c_int32, C.POINTER(_Outputs),
+                                      C.c_int, C.POINTER(C.c_int64)]
     l.fcsim_oracle_philox.restype = None
     l.fcsim_oracle_philox.argtypes = [C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
     l.fcsim_oracle_sample.restype = C.c_int32
@@ -138,7 +141,8 @@ def _p(arr, typ):
     return arr.ctypes.data_as(C.POINTER(typ)) if arr is not None else None
 
 
-def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize, arrcls=False):
+def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize, arrcls=False,
+               mc_mode=0):
     c, keep = marshal(cfg)
     out = {"counters": np.zeros((n, N_COUNTERS), dtype=np.int64)}
     n_rec = n_steps // cfg.trace_stride if cfg.trace_stride > 0 else 0
@@ -154,20 +158,26 @@ def _run_range(cfg, first, n, n_steps, trace, hist, complog, arrlog, admlog_cap,
                  _p(out["complog"], C.c_int32), _p(out["arrlog"], C.c_int32), _p(out["arrcls"], C.c_int32),
                  _p(out["admlog"], C.c_int32),
                  int(admlog_cap), _p(out["n_admlog"], C.c_int64))
-    rc = lib(sanitize).fcsim_oracle_run(C.byref(c), int(first), int(n), int(n_steps), C.byref(o))
+    n_tests = C.c_int64(0)
+    rc = lib(sanitize).fcsim_oracle_run_ex(C.byref(c), int(first), int(n), int(n_steps), C.byref(o), int(mc_mode),
+                                           C.byref(n_tests))
     if rc != 0:
         raise RuntimeError(f"fcsim_oracle_run failed with code {rc}")
     del keep
+    out["n_mc_tests"] = np.array([n_tests.value], dtype=np.int64)
     return out
 
 
 def run(cfg, first_replica=0, n_replicas=None, n_steps=None, *, trace=True, hist=True, complog=True,
-        arrlog=False, admlog_cap=0, threads=1, sanitize=False, arrcls=False):
+        arrlog=False, admlog_cap=0, threads=1, sanitize=False, arrcls=False, mc_mode=0):
     """Simulate replicas [first_replica, first_replica+n_replicas) for slots 1..n_steps.
 
     Returns a dict of numpy arrays: counters [n,28] int64, and (when enabled in ``cfg`` and
     requested) trace [n, n_steps//stride, 2], hist [n, bins], complog [n, cap, 2]; diagnostic
     arrlog [n, n_steps] and admlog [n, admlog_cap, 4] with n_admlog [n].
+    ``mc_mode``: evaluation of the MC benchmark's future-memory test (Section 4.1): 0 = every future slot is
+    summed (the definition, default), 1 = only the last slots of the requests (shortcut), 2 = both, failing
+    on the first disagreement; ``n_mc_tests`` in the result counts the tests made (one entry per thread).
     """
     total = sum(g.n_replicas for g in cfg.groups)
     if n_replicas is None:
@@ -177,11 +187,11 @@ def run(cfg, first_replica=0, n_replicas=None, n_steps=None, *, trace=True, hist
     threads = max(1, min(int(threads), n_replicas)) if n_replicas > 0 else 1
     if threads == 1:
         return _run_range(cfg, first_replica, n_replicas, n_steps, trace, hist, complog, arrlog,
-                          admlog_cap, sanitize, arrcls)
+                          admlog_cap, sanitize, arrcls, mc_mode)
     bounds = np.linspace(0, n_replicas, threads + 1).astype(np.int64)
     with ThreadPoolExecutor(max_workers=threads) as ex:
         futs = [ex.submit(_run_range, cfg, first_replica + int(bounds[i]), int(bounds[i + 1] - bounds[i]),
-                          n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize, arrcls)
+                          n_steps, trace, hist, complog, arrlog, admlog_cap, sanitize, arrcls, mc_mode)
                 for i in range(threads)]
         parts = [f.result() for f in futs]
     out = {}

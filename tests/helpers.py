@@ -11,13 +11,18 @@ POLICIES = {"flow": wl.POLICY_FLOW, "greedy": wl.POLICY_GREEDY, "chunked": wl.PO
             "alpha": wl.POLICY_ALPHA, "mc": wl.POLICY_MC}
 
 
-def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, ma=0, keep=0, **extra):
-    """Constant arrival count n per slot, constant lengths (l, o)."""
+def degenerate_config(n, l, o, policy, b, K, c, M, T, Qcap=64, Acap=64, replicas=1, ma=0, keep=0, n2=None,
+                      thr0=0, thr1=0, **extra):
+    """Constant arrival count n per slot, constant lengths (l, o).  With ``n2`` the arrival law has two states:
+    n arrivals per slot in state 0, n2 in state 1, switching thresholds (thr0, thr1)."""
     pol = POLICIES[policy] if isinstance(policy, str) else policy
+    arrivals = wl.Arrivals((wl.constant_table(n),))
+    if n2 is not None:
+        arrivals = wl.Arrivals((wl.constant_table(n), wl.constant_table(n2)), (int(thr0), int(thr1)))
     return wl.SimConfig(
         M=M, K=K, T_max=T, Qcap=Qcap, Acap=Acap, seed=extra.pop("seed", 7),
         class_law=wl.constant_table(0), prompt=(wl.constant_table(l),), decode=(wl.constant_table(o),),
-        arrivals=(wl.Arrivals((wl.constant_table(n),)),),
+        arrivals=(arrivals,),
         groups=(wl.Group(pol, b_fp=wl.b_to_fp(b), chunk=c, n_replicas=replicas, m_admit=ma, preempt_keep=keep),),
         trace_stride=1, hist_bins=extra.pop("hist_bins", 16), hist_shift=0, complog_cap=4 * T, **extra)
 

@@ -137,3 +137,28 @@ def test_mc_worst_case_projection_equals_known_lengths_when_lengths_are_constant
     k = orc.run(var.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=3, mc_worst_case=0),)), complog=False)
     w = orc.run(var.with_(groups=(wl.Group(wl.POLICY_MC, n_replicas=3, mc_worst_case=1),)), complog=False)
     assert (w["counters"][:, I["sum_U"]] < k["counters"][:, I["sum_U"]]).all()
+
+
+def test_mc_last_slot_shortcut_agrees_with_the_slot_by_slot_test_on_every_decision():
+    # Section 4.1: a request starts only if the usage of EVERY future slot stays within M.  The checker sums
+    # every future slot (mode 0); its opt-in shortcut looks at the requests' last slots only (mode 1).  Mode 2
+    # evaluates both on every admission test and fails on the first disagreement.
+    tests = 0
+    for seed in range(40):
+        cfg = wl.random_medium_config(seed)
+        if not any(g.policy == wl.POLICY_MC for g in cfg.groups):
+            continue
+        both = orc.run(cfg, mc_mode=2, threads=2, trace=False, complog=False)
+        tests += int(both["n_mc_tests"].sum())
+    for seed in range(60):
+        cfg = wl.random_small_config(seed, n_replicas=3, T=97)
+        tests += int(orc.run(cfg, mc_mode=2)["n_mc_tests"].sum())
+    cfg = wl.config6(replicas=1, T=1500)
+    for rate in (5.0, 15.0):
+        c6 = wl.config6(replicas=1, T=1500, total_rate=rate)
+        both = orc.run(c6, mc_mode=2)
+        tests += int(both["n_mc_tests"].sum())
+        fast = orc.run(c6, mc_mode=1)
+        for k in ("counters", "trace", "hist"):
+            assert (both[k] == fast[k]).all()
+    assert tests > 100000, tests
