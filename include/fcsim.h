@@ -130,6 +130,10 @@ typedef struct {
     int32_t hist_bins;    /* 0 = no latency histogram; bin = min(latency >> hist_shift, hist_bins-1) */
     int32_t hist_shift;
     int32_t complog_cap;  /* completions logged per replica; 0 = no log */
+    int32_t trace_bulk;   /* 0 = trace records leave the registers with plain coalesced stores (default, faster as
+                             measured); 1 = they are staged in shared memory and every block of 32 records leaves
+                             with one 256-byte bulk asynchronous copy (needs 512 more bytes of shared memory per
+                             warp).  Same results either way. */
 } fcsim_config;
 
 /* Per-replica counters, all int64, accumulated over the slots run so far (R = number of replicas).
@@ -145,16 +149,27 @@ typedef struct {
         n_logged, q_final, p_final, resid_age, resid_j, mmpp_state;
 } fcsim_counters;
 
+/* Where a summary's p95/p99 come from. */
+enum { FCSIM_PCT_NONE = 0, FCSIM_PCT_HISTOGRAM = 1, FCSIM_PCT_EXACT = 2 };
+
 /* Per-group summary: `total` combines the group's replicas field by field (sum; max for max_lat, max_U,
  * max_Q and steps_done; bitwise or for status).  With n = replicas in the group and T = slots run:
  * mean_latency = sum_lat / completed; mean_utilisation = sum_U / (n T M); request_throughput =
- * completed / (n T); token_throughput = tokens_generated / (n T) (Section 2.2); p95/p99: smallest
- * histogram bin k whose cumulative count reaches ceil(q * completed / 100), reported as
- * ((k+1) << hist_shift) - 1, or max_lat for the open last bin; 0 when there is no histogram or no
- * completion. */
+ * completed / (n T); token_throughput = tokens_generated / (n T) (Section 2.2).
+ * p95/p99 of the end-to-end latency (Section 2.2; the "95% latency" of Section 4.1's figures), q = 95, 99:
+ *  - FCSIM_PCT_EXACT, when there is a completion log and no replica of the group overflowed it: the
+ *    ceil(q * completed / 100)-th smallest latency of the group's completions, selected on the device from
+ *    the log's latency words;
+ *  - FCSIM_PCT_HISTOGRAM otherwise, when there is a histogram: the smallest bin k whose cumulative count
+ *    reaches ceil(q * completed / 100), reported as the bin's largest latency ((k+1) << hist_shift) - 1, or
+ *    max_lat for the open last bin;
+ *  - FCSIM_PCT_NONE (values 0) when nothing completed or neither output exists.
+ * percentile_source says which. */
 typedef struct {
     fcsim_counters total;
     double mean_latency, p95_latency, p99_latency, mean_utilisation, request_throughput, token_throughput;
+    int32_t percentile_source;
+    int32_t reserved;
 } fcsim_summary;
 
 /* DEVICE buffers, caller-owned, each at least the size fcsim_query_sizes reports and 16-byte aligned.
@@ -164,7 +179,8 @@ typedef struct {
  * trace:     [R][T_max / trace_stride] {int32 U_t, int32 |Q_t|}, or NULL when trace_stride = 0.
  * hist:      [R][hist_bins] int32, or NULL when hist_bins = 0.
  * complog:   [R][complog_cap] {int32 t_done, int32 latency}, or NULL when complog_cap = 0.
- * scratch:   per-group reduction area used by fcsim_stats (opaque). */
+ * scratch:   per-group reduction area used by fcsim_stats (opaque; with a completion log it includes the digit
+ *            counts of the percentile selection, 3 * 4096 + 8 words of 8 bytes per group). */
 typedef struct {
     void* workspace;
     void* counters;
@@ -222,7 +238,8 @@ int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_out, fcsim_s
  * device or host allocator and frees nothing.
  *
  * per_group_out: HOST, [n_groups], receives exactly what fcsim_stats would write there.
- * Limit: n_groups * (28 + hist_bins) must not exceed FCSIM_NOALLOC_SCRATCH_WORDS, otherwise
+ * Limit: n_groups * (28 + hist_bins), or n_groups * (28 + hist_bins + 8 + 3 * 4096) with a completion log (the
+ * digit counts of the percentile selection), must not exceed FCSIM_NOALLOC_SCRATCH_WORDS, otherwise
  * FCSIM_ETOOBIG is returned and nothing is launched.
  * First call on a device: the library looks up the device address of its array (one runtime query, no
  * allocation) and remembers it; make that first call outside any stream capture, with the handle's

@@ -214,8 +214,21 @@ def percentile_from_hist(hist64, n, q, shift, max_lat):
     return float(((k + 1) << shift) - 1)
 
 
-def summarize(cfg, counters, hist, n_steps):
-    """Per-group int64 sums and fp64 summaries; ``counters``/``hist`` cover all replicas."""
+def percentile_from_latencies(latencies, q):
+    """The ceil(q*n/100)-th smallest of the n latencies (1-based rank), by a plain sort."""
+    lat = np.sort(np.asarray(latencies, dtype=np.int64))
+    n = lat.shape[0]
+    if n == 0:
+        return 0.0
+    target = (q * n + 99) // 100
+    return float(lat[target - 1])
+
+
+def summarize(cfg, counters, hist, n_steps, complog=None):
+    """Per-group int64 sums and fp64 summaries; ``counters``/``hist``/``complog`` cover all replicas.
+    Tail latencies (Section 2.2 latency; the "95% latency" of Section 4.1): with a completion log that no replica
+    of the group overflowed, the exact order statistic of the logged latencies (percentile_source 2); otherwise
+    from the group's histogram (1); 0 when nothing completed or neither exists (0)."""
     res = []
     first = 0
     for g in cfg.groups:
@@ -239,13 +252,21 @@ def summarize(cfg, counters, hist, n_steps):
         s["mean_utilisation"] = sums["sum_U"] / (float(n) * T * cfg.M) if T > 0 else 0.0
         s["request_throughput"] = done / (float(n) * T) if T > 0 else 0.0
         s["token_throughput"] = sums["tokens_generated"] / (float(n) * T) if T > 0 else 0.0
-        if hist is not None and cfg.hist_bins > 0:
+        s["p95_latency"] = 0.0
+        s["p99_latency"] = 0.0
+        s["percentile_source"] = 0
+        if complog is not None and cfg.complog_cap > 0 and done > 0 and not (sums["status"] & 2):
+            n_log = blk[:, CIDX["n_logged"]]
+            lats = np.concatenate([complog[first + r, :n_log[r], 1] for r in range(g.n_replicas)])
+            assert lats.shape[0] == done
+            s["p95_latency"] = percentile_from_latencies(lats, 95)
+            s["p99_latency"] = percentile_from_latencies(lats, 99)
+            s["percentile_source"] = 2
+        elif hist is not None and cfg.hist_bins > 0 and done > 0:
             h = hist[first:first + g.n_replicas].astype(np.int64).sum(axis=0)
             s["p95_latency"] = percentile_from_hist(h, done, 95, cfg.hist_shift, sums["max_lat"])
             s["p99_latency"] = percentile_from_hist(h, done, 99, cfg.hist_shift, sums["max_lat"])
-        else:
-            s["p95_latency"] = 0.0
-            s["p99_latency"] = 0.0
+            s["percentile_source"] = 1
         res.append(s)
         first += g.n_replicas
     return res

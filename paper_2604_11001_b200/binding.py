@@ -48,7 +48,7 @@ class fcsim_config(C.Structure):
                 ("decode", C.POINTER(fcsim_table)), ("n_arrivals", C.c_int32),
                 ("arrivals", C.POINTER(fcsim_arrivals)), ("n_groups", C.c_int32),
                 ("groups", C.POINTER(fcsim_group)), ("trace_stride", C.c_int32), ("hist_bins", C.c_int32),
-                ("hist_shift", C.c_int32), ("complog_cap", C.c_int32)]
+                ("hist_shift", C.c_int32), ("complog_cap", C.c_int32), ("trace_bulk", C.c_int32)]
 
 
 class fcsim_counters(C.Structure):
@@ -56,7 +56,21 @@ class fcsim_counters(C.Structure):
 
 
 class fcsim_summary(C.Structure):
-    _fields_ = [("total", fcsim_counters)] + [(n, C.c_double) for n in SUMMARY_FLOATS]
+    _fields_ = ([("total", fcsim_counters)] + [(n, C.c_double) for n in SUMMARY_FLOATS]
+                + [("percentile_source", C.c_int32), ("reserved", C.c_int32)])
+
+
+PCT_NONE, PCT_HISTOGRAM, PCT_EXACT = 0, 1, 2
+
+
+def _summary_dicts(summ):
+    out = []
+    for s in summ:
+        d = {n: int(getattr(s.total, n)) for n in COUNTER_NAMES}
+        d.update({n: float(getattr(s, n)) for n in SUMMARY_FLOATS})
+        d["percentile_source"] = int(s.percentile_source)
+        out.append(d)
+    return out
 
 
 class fcsim_buffers(C.Structure):
@@ -168,7 +182,7 @@ def marshal_config(cfg):
     c = fcsim_config(int(cfg.M), int(cfg.K), int(cfg.T_max), int(cfg.Qcap), int(cfg.Acap), int(cfg.seed),
                      len(cfg.prompt), _mk_table(cfg.class_law, keep), prompt, decode, len(cfg.arrivals), arrs,
                      len(cfg.groups), groups, int(cfg.trace_stride), int(cfg.hist_bins), int(cfg.hist_shift),
-                     int(cfg.complog_cap))
+                     int(cfg.complog_cap), int(getattr(cfg, "trace_bulk", 0)))
     keep += [prompt, decode, arrs, groups]
     return c, keep
 
@@ -212,14 +226,7 @@ def fcsim_stats(handle: int, n_replicas: int, n_groups: int, stream=None, want_c
     _check(load().fcsim_stats(C.c_void_p(handle), _stream_ptr(stream),
                               cnt.ctypes.data_as(C.POINTER(fcsim_counters)) if want_counters else None,
                               summ), "fcsim_stats", handle)
-    out = None
-    if want_summary:
-        out = []
-        for s in summ:
-            d = {n: int(getattr(s.total, n)) for n in COUNTER_NAMES}
-            d.update({n: float(getattr(s, n)) for n in SUMMARY_FLOATS})
-            out.append(d)
-    return cnt, out
+    return cnt, (_summary_dicts(summ) if want_summary else None)
 
 
 def fcsim_stats_noalloc(handle: int, n_groups: int, stream=None):
@@ -228,12 +235,7 @@ def fcsim_stats_noalloc(handle: int, n_groups: int, stream=None):
     The group rows use a fixed 1 MiB array inside the library, shared by all calls: do not overlap calls."""
     summ = (fcsim_summary * n_groups)()
     _check(load().fcsim_stats_noalloc(C.c_void_p(handle), _stream_ptr(stream), summ), "fcsim_stats_noalloc", handle)
-    out = []
-    for s in summ:
-        d = {n: int(getattr(s.total, n)) for n in COUNTER_NAMES}
-        d.update({n: float(getattr(s, n)) for n in SUMMARY_FLOATS})
-        out.append(d)
-    return out
+    return _summary_dicts(summ)
 
 
 def fcsim_destroy(handle: int) -> None:
@@ -301,11 +303,7 @@ def fcsim_simulate_host(cfg, n_steps: Optional[int] = None, trace=True, hist=Tru
     _check(load().fcsim_simulate_host(C.byref(c), n_steps, out["counters"].ctypes.data_as(C.POINTER(fcsim_counters)),
                                       ptr(out["trace"]), ptr(out["hist"]), ptr(out["complog"]), summ),
            "fcsim_simulate_host")
-    out["summary"] = []
-    for s in summ:
-        d = {n: int(getattr(s.total, n)) for n in COUNTER_NAMES}
-        d.update({n: float(getattr(s, n)) for n in SUMMARY_FLOATS})
-        out["summary"].append(d)
+    out["summary"] = _summary_dicts(summ)
     return out
 
 

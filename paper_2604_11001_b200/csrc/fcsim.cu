@@ -19,10 +19,11 @@ static_assert(sizeof(fcsim_counters) == C_COUNT * sizeof(int64_t), "counter bloc
 namespace {
 
 constexpr size_t kSmemBudget = 227 * 1024;   // shared memory one CTA may opt in to
-constexpr int kMaxStepsPerLaunch = 32768;    // keeps the 32-bit per-launch partial sums exact
+constexpr int kMaxStepsPerLaunch = 32768;    // upper limit of the slots of one launch (see max_steps_per_launch)
 constexpr long long kTargetWorkPerLaunch = 1LL << 31;  // replica-steps per launch (bounds launch time)
 constexpr uint64_t kGuideMaxRecords = 16384;  // per table: 256 KB of 16-byte records
 constexpr int kStatsChunk = 256;             // replicas reduced by one block before it touches the group row
+constexpr int kSelChunk = 8;                 // replicas whose completion logs one CTA counts before it moves on
 
 struct Layout {
     int Apad, S;
@@ -38,6 +39,22 @@ struct Layout {
 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Exact latency percentiles from the completion log: two-digit selection over the latency words (< 2^24 because
+// the horizon is): a count per value of the high 12 bits, then, for each of the two percentiles, a count per
+// value of the low 12 bits among the latencies whose high bits are the selected ones.
+constexpr int kSelBits = 12, kSelBins = 1 << kSelBits;
+constexpr int kSelResultWords = 8;  // per group: logged completions, p95, p99 (rest unused)
+
+// The per-group reduction area, in 64-bit words: [G][C_COUNT] counter rows, [G][bins] histogram rows and, with a
+// completion log, [G][kSelResultWords] selection results, [G][kSelBins] high-digit counts, [G][2][kSelBins]
+// low-digit counts.  Only the first three parts travel to the host.
+size_t scratch_words(size_t G, size_t bins, int complog_cap) {
+    return G * ((size_t)C_COUNT + bins + (complog_cap > 0 ? (size_t)kSelResultWords + 3 * (size_t)kSelBins : 0));
+}
+size_t scratch_words_to_host(size_t G, size_t bins, int complog_cap) {
+    return G * ((size_t)C_COUNT + bins + (complog_cap > 0 ? (size_t)kSelResultWords : 0));
+}
 
 bool table_ok(const fcsim_table& t, int64_t vmin_lo, int64_t vmax_hi) {
     if (t.n == 0 || t.cdf == nullptr) return false;
@@ -117,12 +134,12 @@ int plan(const fcsim_config* c, Layout* L) {
     L->qcnt_off = L->qwin_off + 64 * 8;
     L->smem_per_warp = L->qcnt_off + (any_classflow ? align_up((size_t)c->n_classes * 4, 16) : 0);
     if (!any_classflow) L->qcnt_off = 0;
-    // Optional trace staging (environment FCSIM_TRACE_BULK=1): 2 x 32 records of 8 bytes in shared memory,
+    // Optional trace staging (fcsim_config::trace_bulk = 1): 2 x 32 records of 8 bytes in shared memory,
     // each full block leaving with one 256-byte bulk copy.  Off by default: measured slower than keeping
     // the records in registers (the stream is 8 bytes per slot, and the extra shared memory costs a CTA).
     L->tstage_off = 0;
-    const char* tb = getenv("FCSIM_TRACE_BULK");
-    if (c->trace_stride > 0 && tb && tb[0] == '1') {
+    if (c->trace_bulk < 0 || c->trace_bulk > 1) return FCSIM_EINVAL;
+    if (c->trace_stride > 0 && c->trace_bulk == 1) {
         L->tstage_off = L->smem_per_warp;
         L->smem_per_warp += 512;
     }
@@ -141,7 +158,7 @@ void sizes_of(const fcsim_config* c, const Layout& L, fcsim_sizes* s) {
     s->trace = (size_t)L.R * (size_t)L.n_rec * 8;
     s->hist = (size_t)L.R * (size_t)c->hist_bins * 4;
     s->complog = (size_t)L.R * (size_t)c->complog_cap * 8;
-    s->scratch = (size_t)c->n_groups * ((size_t)C_COUNT + (size_t)c->hist_bins) * 8;
+    s->scratch = scratch_words(c->n_groups, c->hist_bins, c->complog_cap) * 8;
 }
 
 // ---- statistics kernels ---------------------------------------------------------------------------
@@ -254,6 +271,133 @@ void launch_reduce_hist(const int* hist, const DevGroup* groups, int G, int R, i
         reduce_hist_kernel<4><<<blocks, std::min(256, bins / 4), 0, st>>>(hist, groups, G, R, bins, kStatsChunk, out);
     else
         reduce_hist_kernel<1><<<blocks, 256, 0, st>>>(hist, groups, G, R, bins, kStatsChunk, out);
+}
+
+// ---- exact percentiles from the completion log ---------------------------------------------------------
+// HBM-bound: every logged {slot, latency} pair is read once per pass (8 bytes per completion).
+// One CTA walks chunks of replicas; the counts of the current group are kept in shared memory (32-bit: a chunk
+// holds far fewer than 2^32 records) and flushed into the group's 64-bit row when the group changes.  Lanes of a
+// warp that hit the same bin are combined first (__match_any_sync), because latencies cluster.
+// kPass 1: bin = latency >> 12.  kPass 2: sel[g] = {high digit of p95, of p99}; a latency with that high digit
+// counts under its low 12 bits in the first, respectively second, table of its group.
+template <int kPass>
+__global__ void __launch_bounds__(256) latency_digit_kernel(const int2* __restrict__ complog,
+                                                            const long long* __restrict__ counters,
+                                                            const DevGroup* __restrict__ groups, int n_groups,
+                                                            int n_replicas, int cap, int chunk,
+                                                            const long long* __restrict__ sel,
+                                                            unsigned long long* __restrict__ out) {
+    constexpr int kTables = kPass == 1 ? 1 : 2;
+    __shared__ unsigned int sh[kTables * kSelBins];
+    const int n_chunks = (n_replicas + chunk - 1) / chunk;
+    for (int i = threadIdx.x; i < kTables * kSelBins; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    auto flush = [&](int g) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < kTables * kSelBins; i += blockDim.x) {
+            const unsigned int v = sh[i];
+            if (v) {
+                atomicAdd(out + (size_t)g * kTables * kSelBins + i, (unsigned long long)v);
+                sh[i] = 0;
+            }
+        }
+        __syncthreads();
+    };
+    auto count = [&](unsigned int* table, bool mine, unsigned int bin) {
+        const unsigned int voters = __ballot_sync(0xffffffffu, mine);
+        if (mine) {
+            const unsigned int peers = __match_any_sync(voters, bin);
+            if ((threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(table + bin, (unsigned)__popc(peers));
+        }
+    };
+    for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+        const int r0 = c * chunk, r1 = min(n_replicas, r0 + chunk);
+        int g = group_of(groups, n_groups, r0);
+        int g_end = groups[g].first + groups[g].n;
+        unsigned int hi95 = 0, hi99 = 0;
+        if (kPass == 2) { hi95 = (unsigned)sel[(size_t)g * kSelResultWords + 3]; hi99 = (unsigned)sel[(size_t)g * kSelResultWords + 5]; }
+        for (int r = r0; r < r1; ++r) {
+            if (r >= g_end) {
+                flush(g);
+                ++g;
+                g_end = groups[g].first + groups[g].n;
+                if (kPass == 2) { hi95 = (unsigned)sel[(size_t)g * kSelResultWords + 3]; hi99 = (unsigned)sel[(size_t)g * kSelResultWords + 5]; }
+            }
+            const int n = min((int)counters[(size_t)r * C_COUNT + C_N_LOGGED], cap);
+            const int2* __restrict__ row = complog + (size_t)r * cap;
+            // every thread of the CTA runs the same number of iterations (warp-wide votes inside)
+            for (int base = 0; base < n; base += 4 * (int)blockDim.x) {
+                int lat[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {  // four independent loads in flight
+                    const int i = base + u * (int)blockDim.x + (int)threadIdx.x;
+                    lat[u] = i < n ? __ldg(row + i).y : -1;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool have = lat[u] >= 0;
+                    const unsigned int v = (unsigned)lat[u] & 0xffffffu;
+                    if (kPass == 1) {
+                        count(sh, have, v >> kSelBits);
+                    } else {
+                        count(sh, have && (v >> kSelBits) == hi95, v & (kSelBins - 1));
+                        count(sh + kSelBins, have && (v >> kSelBits) == hi99, v & (kSelBins - 1));
+                    }
+                }
+            }
+        }
+        flush(g);
+    }
+}
+
+// One CTA of 256 threads per group: the smallest bin whose cumulative count reaches a target rank.
+// kPass 1: row = the group's high-digit counts; total = their sum; targets ceil(95 total / 100) and ceil(99 total / 100);
+//          res[g] = {total, 0, 0, bin95, rank95 within that bin, bin99, rank99 within that bin, 0}.
+// kPass 2: rows = the group's two low-digit tables, targets = the ranks left by pass 1;
+//          res[g][1] = p95 and res[g][2] = p99 (high digit << 12 | low digit).
+template <int kPass>
+__global__ void __launch_bounds__(256) latency_select_kernel(const unsigned long long* __restrict__ tables,
+                                                             long long* __restrict__ res) {
+    __shared__ unsigned long long part[256];
+    __shared__ unsigned long long total_s;
+    const int g = blockIdx.x, tid = threadIdx.x;
+    constexpr int kPer = kSelBins / 256;
+    long long* out = res + (size_t)g * kSelResultWords;
+    for (int qi = 0; qi < 2; ++qi) {
+        const unsigned long long* row = tables + ((size_t)g * (kPass == 1 ? 1 : 2) + (kPass == 1 ? 0 : qi)) * kSelBins;
+        unsigned long long mine = 0;
+        for (int k = 0; k < kPer; ++k) mine += row[tid * kPer + k];
+        part[tid] = mine;
+        __syncthreads();
+        if (tid == 0) {  // 256 partial sums: a serial scan is short next to the pass over the log
+            unsigned long long run = 0;
+            for (int k = 0; k < 256; ++k) { const unsigned long long v = part[k]; part[k] = run; run += v; }
+            total_s = run;
+        }
+        __syncthreads();
+        const unsigned long long total = total_s;
+        unsigned long long target;
+        if (kPass == 1) target = ((unsigned long long)(qi == 0 ? 95 : 99) * total + 99) / 100;
+        else target = (unsigned long long)out[4 + 2 * qi];
+        if (total > 0 && target > 0 && part[tid] < target && part[tid] + mine >= target) {
+            unsigned long long cum = part[tid];
+            for (int k = 0; k < kPer; ++k) {
+                const unsigned long long v = row[tid * kPer + k];
+                if (cum + v >= target) {
+                    if (kPass == 1) {
+                        out[3 + 2 * qi] = tid * kPer + k;
+                        out[4 + 2 * qi] = (long long)(target - cum);
+                    } else {
+                        out[1 + qi] = (out[3 + 2 * qi] << kSelBits) | (long long)(tid * kPer + k);
+                    }
+                    break;
+                }
+                cum += v;
+            }
+        }
+        if (kPass == 1 && qi == 0 && tid == 0) out[0] = (long long)total;
+        __syncthreads();
+    }
 }
 
 }  // namespace
@@ -672,10 +816,21 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     return FCSIM_OK;
 }
 
+// Slots of one launch.  Bounded by the work of a launch (its duration) and by the 32-bit partial sums that the
+// step kernel keeps per launch and folds into the 64-bit counters at its end.  With n slots per launch:
+//   sum of |P| + |Q| per slot          <= (Qcap + 2 Acap) n      (the queue may hold Qcap + Acap after evictions)
+//   tokens generated, completions      <= Acap n
+//   arrivals                           <= 255 n
+//   output lengths of the completions, per lane <= Acap n + M    (tokens made in the launch plus those the
+//                                                                 requests running at its start already held)
+// so n <= (2^32 - 2^30 - 1) / (Qcap + 2 Acap) keeps all of them exact (M <= 2^30); with Qcap + Acap <= 2^20 that
+// is at least 1536 slots.
 static int max_steps_per_launch(const fcsim* h) {
     long long s = kTargetWorkPerLaunch / std::max<long long>(1, h->L.R);
     s = std::max<long long>(256, std::min<long long>(s, kMaxStepsPerLaunch));
-    return (int)s;
+    const long long per_slot = (long long)h->cfg.Qcap + 2LL * h->cfg.Acap;
+    s = std::min<long long>(s, ((1LL << 32) - (1LL << 30) - 1) / per_slot);
+    return (int)std::max<long long>(1, s);
 }
 
 extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
@@ -730,59 +885,105 @@ static double percentile(const long long* hist, int bins, int shift, long long n
     return (double)((((long long)k + 1) << shift) - 1);
 }
 
+// The group rows of a statistics call: cleared, reduced on the device into `d_rows` (layout: scratch_words) and
+// the part the host needs copied to `host_rows`, all on `st`.  Nothing is allocated here.
+static int reduce_groups(fcsim* h, cudaStream_t st, long long* d_rows, long long* host_rows) {
+    const int G = (int)h->groups.size();
+    const int bins = h->cfg.hist_bins;
+    const int R = (int)h->L.R;
+    const bool with_log = h->cfg.complog_cap > 0;
+    long long* d_cnt = d_rows;
+    long long* d_hist = d_cnt + (size_t)G * C_COUNT;
+    long long* d_res = d_hist + (size_t)G * bins;
+    unsigned long long* d_hi = reinterpret_cast<unsigned long long*>(d_res + (size_t)G * kSelResultWords);
+    unsigned long long* d_lo = d_hi + (size_t)G * kSelBins;
+    // the area still holds the rows of the previous call: the sums must start from zero
+    CUDA_TRY(h, cudaMemsetAsync(d_rows, 0, scratch_words(G, bins, h->cfg.complog_cap) * 8, st));
+    const int n_chunks = (R + kStatsChunk - 1) / kStatsChunk;
+    {
+        const int warps_per_block = 8;
+        const int blocks = std::max(1, std::min((n_chunks + warps_per_block - 1) / warps_per_block, h->sm_count * 8));
+        reduce_counters_kernel<<<blocks, warps_per_block * 32, 0, st>>>(
+            static_cast<const long long*>(h->buf.counters), h->d_groups, G, R, kStatsChunk, d_cnt);
+        CUDA_TRY(h, cudaGetLastError());
+    }
+    if (bins > 0) {
+        const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
+        launch_reduce_hist(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins, blocks, d_hist, st);
+        CUDA_TRY(h, cudaGetLastError());
+    }
+    if (with_log) {
+        const int chunk = kSelChunk;
+        const int blocks = std::max(1, std::min((R + chunk - 1) / chunk, h->sm_count * 8));
+        const int2* log = static_cast<const int2*>(h->buf.complog);
+        const long long* cnt = static_cast<const long long*>(h->buf.counters);
+        latency_digit_kernel<1><<<blocks, 256, 0, st>>>(log, cnt, h->d_groups, G, R, h->cfg.complog_cap, chunk, d_res, d_hi);
+        CUDA_TRY(h, cudaGetLastError());
+        latency_select_kernel<1><<<G, 256, 0, st>>>(d_hi, d_res);
+        CUDA_TRY(h, cudaGetLastError());
+        latency_digit_kernel<2><<<blocks, 256, 0, st>>>(log, cnt, h->d_groups, G, R, h->cfg.complog_cap, chunk, d_res, d_lo);
+        CUDA_TRY(h, cudaGetLastError());
+        latency_select_kernel<2><<<G, 256, 0, st>>>(d_lo, d_res);
+        CUDA_TRY(h, cudaGetLastError());
+    }
+    CUDA_TRY(h, cudaMemcpyAsync(host_rows, d_rows, scratch_words_to_host(G, bins, h->cfg.complog_cap) * 8,
+                                cudaMemcpyDeviceToHost, st));
+    return FCSIM_OK;
+}
+
+// Per-group summaries from the reduced rows (host arithmetic: one division per figure).
+static void fill_summaries(const fcsim* h, const long long* rows, fcsim_summary* per_group_out) {
+    const int G = (int)h->groups.size();
+    const int bins = h->cfg.hist_bins;
+    const double T = (double)h->t_done;
+    const long long* res = rows + (size_t)G * ((size_t)C_COUNT + bins);
+    for (int g = 0; g < G; ++g) {
+        fcsim_summary& s = per_group_out[g];
+        std::memcpy(&s.total, rows + (size_t)g * C_COUNT, sizeof(fcsim_counters));
+        const double n = (double)h->groups[g].n_replicas;
+        const fcsim_counters& c = s.total;
+        s.mean_latency = c.completed > 0 ? (double)c.sum_lat / (double)c.completed : 0.0;
+        s.mean_utilisation = T > 0 ? (double)c.sum_U / (n * T * (double)h->cfg.M) : 0.0;
+        s.request_throughput = T > 0 ? (double)c.completed / (n * T) : 0.0;
+        s.token_throughput = T > 0 ? (double)c.tokens_generated / (n * T) : 0.0;
+        s.percentile_source = FCSIM_PCT_NONE;
+        s.reserved = 0;
+        s.p95_latency = s.p99_latency = 0.0;
+        const long long* sel = res + (size_t)g * kSelResultWords;
+        if (h->cfg.complog_cap > 0 && c.completed > 0 && (c.status & 2) == 0 && sel[0] == c.completed) {
+            // every completion of the group is in the log: the order statistics themselves
+            s.p95_latency = (double)sel[1];
+            s.p99_latency = (double)sel[2];
+            s.percentile_source = FCSIM_PCT_EXACT;
+        } else if (bins > 0 && c.completed > 0) {
+            const long long* gh = rows + (size_t)G * C_COUNT + (size_t)g * bins;
+            s.p95_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 95, c.max_lat);
+            s.p99_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 99, c.max_lat);
+            s.percentile_source = FCSIM_PCT_HISTOGRAM;
+        }
+    }
+}
+
 extern "C" int fcsim_stats(fcsim_t* h, void* cuda_stream, fcsim_counters* host_out, fcsim_summary* per_group_out) {
     if (!h) return FCSIM_EINVAL;
     if (int rc = check_device(h)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int G = (int)h->groups.size();
-    const int bins = h->cfg.hist_bins;
     const int R = (int)h->L.R;
-    std::vector<long long> host_scratch;
+    std::vector<long long> host_rows;
     if (per_group_out) {
-        long long* d_cnt = static_cast<long long*>(h->buf.scratch);
-        long long* d_hist = d_cnt + (size_t)G * C_COUNT;
-        const size_t bytes = (size_t)G * ((size_t)C_COUNT + bins) * 8;
-        CUDA_TRY(h, cudaMemsetAsync(h->buf.scratch, 0, bytes, st));
-        const int n_chunks = (R + kStatsChunk - 1) / kStatsChunk;
-        {
-            const int warps_per_block = 8;
-            const int blocks = std::max(1, std::min((n_chunks + warps_per_block - 1) / warps_per_block, h->sm_count * 8));
-            reduce_counters_kernel<<<blocks, warps_per_block * 32, 0, st>>>(
-                static_cast<const long long*>(h->buf.counters), h->d_groups, G, R, kStatsChunk, d_cnt);
-            CUDA_TRY(h, cudaGetLastError());
-        }
-        if (bins > 0) {
-            const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
-            launch_reduce_hist(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins, blocks, d_hist, st);
-            CUDA_TRY(h, cudaGetLastError());
-        }
         try {
-            host_scratch.resize(bytes / 8);
+            host_rows.resize(scratch_words_to_host(G, h->cfg.hist_bins, h->cfg.complog_cap));
         } catch (...) {
             return FCSIM_ENOMEM;
         }
-        CUDA_TRY(h, cudaMemcpyAsync(host_scratch.data(), h->buf.scratch, bytes, cudaMemcpyDeviceToHost, st));
+        if (int rc = reduce_groups(h, st, static_cast<long long*>(h->buf.scratch), host_rows.data())) return rc;
     }
     if (host_out)
         CUDA_TRY(h, cudaMemcpyAsync(host_out, h->buf.counters, (size_t)R * sizeof(fcsim_counters),
                                     cudaMemcpyDeviceToHost, st));
     CUDA_TRY(h, cudaStreamSynchronize(st));
-    if (per_group_out) {
-        const double T = (double)h->t_done;
-        for (int g = 0; g < G; ++g) {
-            fcsim_summary& s = per_group_out[g];
-            std::memcpy(&s.total, host_scratch.data() + (size_t)g * C_COUNT, sizeof(fcsim_counters));
-            const double n = (double)h->groups[g].n_replicas;
-            const fcsim_counters& c = s.total;
-            s.mean_latency = c.completed > 0 ? (double)c.sum_lat / (double)c.completed : 0.0;
-            s.mean_utilisation = T > 0 ? (double)c.sum_U / (n * T * (double)h->cfg.M) : 0.0;
-            s.request_throughput = T > 0 ? (double)c.completed / (n * T) : 0.0;
-            s.token_throughput = T > 0 ? (double)c.tokens_generated / (n * T) : 0.0;
-            const long long* gh = host_scratch.data() + (size_t)G * C_COUNT + (size_t)g * bins;
-            s.p95_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 95, c.max_lat);
-            s.p99_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 99, c.max_lat);
-        }
-    }
+    if (per_group_out) fill_summaries(h, host_rows.data(), per_group_out);
     return FCSIM_OK;
 }
 
@@ -801,9 +1002,7 @@ static long long* g_noalloc_dev_ptr[kNoallocMaxDevices] = {nullptr};
 extern "C" int fcsim_stats_noalloc(fcsim_t* h, void* cuda_stream, fcsim_summary* per_group_out) {
     if (!h || !per_group_out) return FCSIM_EINVAL;
     const int G = (int)h->groups.size();
-    const int bins = h->cfg.hist_bins;
-    const int R = (int)h->L.R;
-    const size_t words = (size_t)G * ((size_t)C_COUNT + (size_t)bins);
+    const size_t words = scratch_words(G, h->cfg.hist_bins, h->cfg.complog_cap);
     if (words > (size_t)FCSIM_NOALLOC_SCRATCH_WORDS) return FCSIM_ETOOBIG;
     int dev = -1;
     CUDA_TRY(h, cudaGetDevice(&dev));
@@ -814,39 +1013,9 @@ extern "C" int fcsim_stats_noalloc(fcsim_t* h, void* cuda_stream, fcsim_summary*
         g_noalloc_dev_ptr[dev] = static_cast<long long*>(sym);
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    long long* d_cnt = g_noalloc_dev_ptr[dev];
-    long long* d_hist = d_cnt + (size_t)G * C_COUNT;
-    // the array still holds the rows of the previous call: the sums must start from zero
-    CUDA_TRY(h, cudaMemsetAsync(d_cnt, 0, words * 8, st));
-    const int n_chunks = (R + kStatsChunk - 1) / kStatsChunk;
-    {
-        const int warps_per_block = 8;
-        const int blocks = std::max(1, std::min((n_chunks + warps_per_block - 1) / warps_per_block, h->sm_count * 8));
-        reduce_counters_kernel<<<blocks, warps_per_block * 32, 0, st>>>(
-            static_cast<const long long*>(h->buf.counters), h->d_groups, G, R, kStatsChunk, d_cnt);
-        CUDA_TRY(h, cudaGetLastError());
-    }
-    if (bins > 0) {
-        const int blocks = std::max(1, std::min(n_chunks, h->sm_count * 16));
-        launch_reduce_hist(static_cast<const int*>(h->buf.hist), h->d_groups, G, R, bins, blocks, d_hist, st);
-        CUDA_TRY(h, cudaGetLastError());
-    }
-    CUDA_TRY(h, cudaMemcpyAsync(g_noalloc_host_rows, d_cnt, words * 8, cudaMemcpyDeviceToHost, st));
+    if (int rc = reduce_groups(h, st, g_noalloc_dev_ptr[dev], g_noalloc_host_rows)) return rc;
     CUDA_TRY(h, cudaStreamSynchronize(st));
-    const double T = (double)h->t_done;
-    for (int g = 0; g < G; ++g) {
-        fcsim_summary& s = per_group_out[g];
-        std::memcpy(&s.total, g_noalloc_host_rows + (size_t)g * C_COUNT, sizeof(fcsim_counters));
-        const double n = (double)h->groups[g].n_replicas;
-        const fcsim_counters& c = s.total;
-        s.mean_latency = c.completed > 0 ? (double)c.sum_lat / (double)c.completed : 0.0;
-        s.mean_utilisation = T > 0 ? (double)c.sum_U / (n * T * (double)h->cfg.M) : 0.0;
-        s.request_throughput = T > 0 ? (double)c.completed / (n * T) : 0.0;
-        s.token_throughput = T > 0 ? (double)c.tokens_generated / (n * T) : 0.0;
-        const long long* gh = g_noalloc_host_rows + (size_t)G * C_COUNT + (size_t)g * bins;
-        s.p95_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 95, c.max_lat);
-        s.p99_latency = percentile(gh, bins, h->cfg.hist_shift, c.completed, 99, c.max_lat);
-    }
+    fill_summaries(h, g_noalloc_host_rows, per_group_out);
     return FCSIM_OK;
 }
 

@@ -408,7 +408,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 #define CSET(idx, v) do { const long long v__ = (long long)(v); if (lane == (idx)) cnt = v__; } while (0)
 #define WA(x) ((x) >= Acap ? (x) - Acap : (x))
 
-        // per-launch partial sums of the quantities touched every slot
+        // per-launch partial sums of the quantities touched every slot.  The 32-bit ones cannot wrap because the
+        // host bounds the slots of a launch by (2^32 - 2^30) / (Qcap + 2 Acap): sumN grows by at most
+        // Qcap + 2 Acap per slot, tokgen by at most Acap, arrived and accepted by at most 255.
         unsigned long long sumU = 0;
         uint32_t sumN = 0, tokgen = 0, arrived = 0, accepted = 0;
         int maxU = 0, maxQ = 0;
@@ -420,6 +422,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         bool gate_closed = false;
         bool mc_refused = false;  // MC benchmark: the last future-memory test refused the queue head
         // statistics of completions, private to the lane that saw them; reduced once when the replica is put back
+        // (acc_o: the output lengths of a launch's completions add up to at most the tokens generated in the
+        // launch, <= Acap per slot, plus the tokens the running requests held at its start, <= M <= 2^30)
         unsigned long long acc_lat = 0, acc_w = 0;
         uint32_t acc_o = 0, completed = 0;
         int acc_maxlat = 0;

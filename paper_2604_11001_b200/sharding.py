@@ -10,6 +10,8 @@ from __future__ import annotations
 
 from dataclasses import replace
 
+import torch
+
 MAX_FIELDS = (0, 16, 18, 20)   # steps_done, max_lat, max_U, max_Q combine by maximum
 OR_FIELDS = (1,)               # status combines by bitwise or
 
@@ -37,7 +39,8 @@ def combine_group_totals(totals, dist=None):
         dist.all_reduce(col, op=dist.ReduceOp.MAX)
         out[:, f] = col
     for f in OR_FIELDS:
-        col = totals[:, f].clone()
-        dist.all_reduce(col, op=dist.ReduceOp.BOR)
-        out[:, f] = col
+        # bitwise or as a maximum per bit (status has two bits): every backend implements MAX, NCCL has no BOR
+        bits = ((totals[:, f].unsqueeze(1) >> torch.arange(8, device=totals.device)) & 1).contiguous()
+        dist.all_reduce(bits, op=dist.ReduceOp.MAX)
+        out[:, f] = (bits << torch.arange(8, device=totals.device)).sum(dim=1)
     return out

@@ -188,6 +188,7 @@ class SimConfig:
     hist_bins: int = 0
     hist_shift: int = 0
     complog_cap: int = 0
+    trace_bulk: int = 0        # 1 = trace records staged in shared memory and stored with bulk copies (same results)
     name: str = ""
     notes: dict = field(default_factory=dict, compare=False)
 

@@ -47,12 +47,15 @@ def assert_same(cfg, gpu, ref, n_steps, what=""):
             assert (gpu["complog"][r, :n[r]] == ref["complog"][r, :n[r]]).all(), f"{what} completion log differs (replica {r})"
 
 
-def assert_summary_close(cfg, gpu_summary, counters, hist, n_steps, rtol=1e-9):
-    """fp64 summaries derived from int64 sums: relative 1e-9."""
-    ref = orc.summarize(cfg, counters, hist, n_steps)
+def assert_summary_close(cfg, gpu_summary, counters, hist, n_steps, complog=None, rtol=1e-9):
+    """fp64 summaries derived from int64 sums: relative 1e-9.  With the checker's completion log the tail
+    latencies must be the exact order statistics, and say so."""
+    ref = orc.summarize(cfg, counters, hist, n_steps, complog)
     for g, (a, b) in enumerate(zip(gpu_summary, ref)):
         for k in orc.COUNTER_NAMES:
             assert a[k] == b[k], (g, k, a[k], b[k])
         for k in ("mean_latency", "p95_latency", "p99_latency", "mean_utilisation", "request_throughput",
                   "token_throughput"):
             assert abs(a[k] - b[k]) <= rtol * max(abs(b[k]), 1e-300), (g, k, a[k], b[k])
+        if complog is not None or cfg.complog_cap == 0:
+            assert a["percentile_source"] == b["percentile_source"], (g, a["percentile_source"], b["percentile_source"])

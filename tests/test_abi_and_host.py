@@ -29,7 +29,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_counter_block_is_28_int64():
     assert C.sizeof(fb.fcsim_counters) == 28 * 8
-    assert C.sizeof(fb.fcsim_summary) == 28 * 8 + 6 * 8
+    assert C.sizeof(fb.fcsim_summary) == 28 * 8 + 6 * 8 + 8
     assert fb.COUNTER_NAMES[0] == "steps_done" and fb.COUNTER_NAMES[-1] == "mmpp_state"
 
 

@@ -116,15 +116,15 @@ def test_config2_full():
 
 def test_config3_full():
     cfg = wl.config3()
-    # every 16th group of the 64 x 64 sweep (offset so that rates and flow-control settings both vary), all 16
-    # replicas of each: 4096 replicas over the full horizon
-    groups = range(5, len(cfg.groups), 16)
-    _run_full(cfg, 2000, [16 * g + k for g in groups for k in range(16)])
+    # every 4th group of the 64 x 64 sweep (offset 1: every arrival rate, 16 of the 64 flow-control settings), all
+    # 16 replicas of each: 16 384 replicas over the full horizon
+    groups = range(1, len(cfg.groups), 4)
+    _run_full(cfg, 2000, [16 * g + k for g in groups for k in range(16)], batch=1024)
 
 
 def test_config4_full():
     cfg = wl.config4()
-    _run_full(cfg, 2000, range(1, cfg.n_replicas, 4))      # every 4th replica of both groups
+    _run_full(cfg, 2000, range(cfg.n_replicas), batch=4096)   # every replica of both groups, every output word
 
 
 def test_config5_full():
@@ -134,14 +134,19 @@ def test_config5_full():
     assert c[:, I["dropped"]].min() > 0 and c[:, I["evictions"]].sum() > 0
 
 
-def test_config5_first_2000_slots_every_fourth_replica():
+def test_config5_first_2000_slots_every_replica():
     cfg = wl.config5()
-    _run_full(cfg, 2000, range(0, cfg.n_replicas, 4), n_steps=2000, batch=8192)
+    _run_full(cfg, 2000, range(cfg.n_replicas), n_steps=2000, batch=16384)
 
 
 def test_config6_full_paper_setting():
     cfg = wl.config6()
-    c = _run_full(cfg, 500, _sample(cfg, 8, 6))
+    # 64 replicas of each of the four cheap policies, 24 of each MC group (the checker's future-memory test walks
+    # every future slot of every running request)
+    n0 = cfg.groups[0].n_replicas
+    sample = sorted([g * n0 + k for g in range(4) for k in range(g, n0, n0 // 64)][:4 * 64]
+                    + [g * n0 + k for g in (4, 5) for k in range(g, n0, n0 // 24)][:2 * 24])
+    c = _run_full(cfg, 500, sample)
     # Section 4.1's load is light (about 0.41 of the necessary-condition load): flow control with b = 12 > lambda
     # never overflows, and nothing is dropped
     n = cfg.groups[0].n_replicas

@@ -31,7 +31,7 @@ def test_random_small_configs(seed):
     gpu = run_gpu(cfg)
     ref = orc.run(cfg)
     assert_same(cfg, gpu, ref, cfg.T_max, cfg.name)
-    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max, ref["complog"])
 
 
 @pytest.mark.parametrize("cfg", scaled_presets(), ids=lambda c: c.name)
@@ -39,7 +39,7 @@ def test_scaled_presets(cfg):
     gpu = run_gpu(cfg)
     ref = orc.run(cfg, threads=8)
     assert_same(cfg, gpu, ref, cfg.T_max, cfg.name)
-    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max, ref["complog"])
 
 
 def test_config1_full():
@@ -47,7 +47,7 @@ def test_config1_full():
     gpu = run_gpu(cfg)
     ref = orc.run(cfg, threads=8)
     assert_same(cfg, gpu, ref, cfg.T_max, "cfg1")
-    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max, ref["complog"])
 
 
 @pytest.mark.parametrize("pieces", [[1] * 40 + [60], [33, 31, 36], [7, 64, 29], [99, 1]])
@@ -70,7 +70,7 @@ def test_pause_counters_match_a_shorter_run():
     gpu = run_gpu(cfg, n_steps=1234)
     ref = orc.run(cfg, n_steps=1234)
     assert_same(cfg, gpu, ref, 1234, "cfg5 paused")
-    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 1234)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 1234, ref["complog"])
 
 
 def test_more_replicas_than_resident_warps_and_many_groups():
@@ -80,7 +80,7 @@ def test_more_replicas_than_resident_warps_and_many_groups():
     gpu = run_gpu(cfg)
     ref = orc.run(cfg, threads=8)
     assert_same(cfg, gpu, ref, cfg.T_max, "cfg3 grid")
-    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max, ref["complog"])
     big = wl.config1(replicas=20000, T=64).with_(trace_stride=8, complog_cap=8)
     gpu = run_gpu(big)
     ref = orc.run(big, threads=8)
@@ -120,7 +120,7 @@ def test_host_buffer_entry_point():
     out = fb.fcsim_simulate_host(cfg)
     ref = orc.run(cfg)
     assert_same(cfg, out, ref, 500, "simulate_host")
-    assert_summary_close(cfg, out["summary"], ref["counters"], ref["hist"], 500)
+    assert_summary_close(cfg, out["summary"], ref["counters"], ref["hist"], 500, ref["complog"])
 
 
 def test_large_active_set_and_lazy_removal_paths():
@@ -140,13 +140,12 @@ def test_large_active_set_and_lazy_removal_paths():
     assert_same(churn, run_gpu(churn, pieces=[1000, 1, 1999]), orc.run(churn), 3000, "eviction churn")
 
 
-def test_trace_bulk_copy_variant(monkeypatch):
+def test_trace_bulk_copy_variant():
     # opt-in variant: trace records staged in shared memory and stored with 256-byte bulk copies.  Rows of 333
     # records: odd rows start 8 bytes off a 16-byte boundary and must fall back to plain stores.
-    monkeypatch.setenv("FCSIM_TRACE_BULK", "1")
-    cfg = wl.config1(replicas=9, T=333)
+    cfg = wl.config1(replicas=9, T=333).with_(trace_bulk=1)
     assert_same(cfg, run_gpu(cfg, pieces=[100, 7, 226]), orc.run(cfg), 333, "bulk trace")
-    cfg = wl.config2(replicas=2, T=2000)
+    cfg = wl.config2(replicas=2, T=2000).with_(trace_bulk=1)
     assert_same(cfg, run_gpu(cfg), orc.run(cfg), 2000, "bulk trace cfg2")
 
 
@@ -190,7 +189,10 @@ def test_random_medium_configs(seed):
     cfg = wl.random_medium_config(seed)
     cut = 1 + (seed * 97) % (cfg.T_max - 1)
     ref = orc.run(cfg, threads=4)
-    assert_same(cfg, run_gpu(cfg, pieces=[cut, cfg.T_max - cut]), ref, cfg.T_max, cfg.name)
+    gpu = run_gpu(cfg, pieces=[cut, cfg.T_max - cut])
+    assert_same(cfg, gpu, ref, cfg.T_max, cfg.name)
+    # logs of 300 entries overflow (histogram percentiles), logs of 20 000 do not (exact percentiles)
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], cfg.T_max, ref["complog"])
 
 
 def test_handles_with_different_shared_memory_needs_coexist():
@@ -364,3 +366,55 @@ def test_two_handles_driven_from_two_threads():
     assert not errors, errors
     assert (out["big"] == orc.run(big_cfg)["counters"]).all()
     assert (out["small"] == orc.run(small_cfg)["counters"]).all()
+
+
+def test_exact_percentiles_from_the_completion_log():
+    # the hand trace whose 7th smallest latency is 6 while its histogram bin ends at 7
+    cfg = degenerate_config(n=1, l=2, o=3, policy="flow", b=1, K=0, c=0, M=11, T=12, hist_bins=8).with_(hist_shift=2)
+    s = run_gpu(cfg)["summary"][0]
+    assert s["p95_latency"] == 6.0 and s["p99_latency"] == 6.0 and s["percentile_source"] == 2
+    # groups of unequal size, latencies on both sides of 4096 (two-digit selection), several replicas per group,
+    # p95 and p99 in different high digits; one group completes nothing
+    base = wl.config2(replicas=1, T=9000)
+    groups = (wl.Group(wl.POLICY_FLOW, b_fp=0x6000, n_replicas=37, rng_replica_base=3),
+              wl.Group(wl.POLICY_FLOW, b_fp=0, n_replicas=2),
+              wl.Group(wl.POLICY_GREEDY, n_replicas=11),
+              wl.Group(wl.POLICY_FLOW, b_fp=0x20000, n_replicas=1, rng_replica_base=77))
+    cfg = base.with_(groups=groups, Qcap=4096, trace_stride=0, hist_shift=7, complog_cap=8192)
+    ref = orc.run(cfg, threads=8)
+    want = orc.summarize(cfg, ref["counters"], ref["hist"], 9000, ref["complog"])
+    assert want[0]["max_lat"] > 4096 and want[0]["percentile_source"] == 2 and want[1]["percentile_source"] == 0
+    assert want[0]["p99_latency"] - want[0]["p95_latency"] > 100
+    hist_rule = orc.summarize(cfg, ref["counters"], ref["hist"], 9000)
+    assert hist_rule[0]["p95_latency"] != want[0]["p95_latency"]
+    gpu = run_gpu(cfg, pieces=[4000, 5000])
+    assert_same(cfg, gpu, ref, 9000, "exact percentiles")
+    assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 9000, ref["complog"])
+    # a log too small for the run: the histogram rule, and the summary says so
+    short = cfg.with_(complog_cap=64)
+    refs = orc.run(short, threads=8)
+    gpus = run_gpu(short)
+    assert gpus["summary"][0]["percentile_source"] == 1
+    assert_summary_close(short, gpus["summary"], refs["counters"], refs["hist"], 9000, refs["complog"])
+
+
+def test_standing_queue_of_200000_over_a_long_run():
+    # |P| + |Q| summed over the slots passes 2^32 within what used to be one launch: the per-launch partial sums
+    # are 32-bit, so the library must cut the launches short enough (Qcap + 2 Acap per slot at most).  Nothing is
+    # ever activated (b = 0), so the slot-exact Little identity reads sum_N = resid_age.
+    from paper_2604_11001_b200 import binding as fb
+    cfg = degenerate_config(n=255, l=1, o=1, policy="flow", b=0, K=0, c=0, M=1000, T=33000, Qcap=200000, Acap=64,
+                            replicas=2)
+    cfg = cfg.with_(trace_stride=1000, complog_cap=0, hist_bins=0)
+    sim = fb.Simulation(cfg)
+    per = sim.launch_info()["max_steps_per_launch"]
+    assert per * (200000 + 128) < (1 << 32) - (1 << 30)
+    sim.close()
+    gpu = run_gpu(cfg)
+    c = gpu["counters"]
+    I = orc.CIDX
+    assert (c[:, I["sum_N"]] > (1 << 32)).all() and (c[:, I["sum_lat"]] == 0).all()
+    assert (c[:, I["sum_N"]] == c[:, I["sum_lat"]] + c[:, I["resid_age"]]).all()
+    assert (c[:, I["q_final"]] == 200000).all() and (c[:, I["dropped"]] == 255 * 33000 - 200000).all()
+    ref = orc.run(cfg, threads=2)
+    assert_same(cfg, gpu, ref, 33000, "standing queue")

@@ -96,6 +96,31 @@ def test_percentile_rule_and_summaries():
     assert s["mean_utilisation"] == sum((3, 7, 9, 8, 7, 9, 8, 7, 9, 8, 7, 9)) / (12 * 11)
     # token throughput: tokens generated per slot (Section 2.2)
     assert s["token_throughput"] == out["counters"][0, I["tokens_generated"]] / 12
+    assert s["percentile_source"] == 1
+
+
+def test_exact_percentiles_from_the_completion_log_differ_from_the_bin_edge():
+    # same hand trace with 4-slot histogram bins: latencies 3,3 fall in bin 0 and 4,4,5,5,6 in bin 1, so the
+    # histogram rule reports the edge of bin 1, (2 << 2) - 1 = 7, while the 7th smallest latency itself is 6
+    cfg = degenerate_config(n=1, l=2, o=3, policy="flow", b=1, K=0, c=0, M=11, T=12, hist_bins=8).with_(hist_shift=2)
+    out = orc.run(cfg)
+    assert out["complog"][0, :7, 1].tolist() == [3, 3, 4, 4, 5, 5, 6]
+    by_hist = orc.summarize(cfg, out["counters"], out["hist"], 12)[0]
+    exact = orc.summarize(cfg, out["counters"], out["hist"], 12, out["complog"])[0]
+    assert by_hist["p95_latency"] == 7.0 and by_hist["percentile_source"] == 1
+    assert exact["p95_latency"] == 6.0 and exact["p99_latency"] == 6.0 and exact["percentile_source"] == 2
+    # rank rule ceil(q n / 100), 1-based: 100 distinct values -> the 95th and 99th; 101 values -> ranks 96 and 100
+    rng = np.random.default_rng(0)
+    assert orc.percentile_from_latencies(rng.permutation(np.arange(1, 101)), 95) == 95.0
+    assert orc.percentile_from_latencies(rng.permutation(np.arange(1, 101)), 99) == 99.0
+    assert orc.percentile_from_latencies(rng.permutation(np.arange(1, 102)), 95) == 96.0
+    assert orc.percentile_from_latencies(rng.permutation(np.arange(1, 102)), 99) == 100.0
+    assert orc.percentile_from_latencies([7], 95) == 7.0 and orc.percentile_from_latencies([], 95) == 0.0
+    # a log that overflowed cannot give the order statistics: the histogram rule is used and reported
+    small = cfg.with_(complog_cap=3)
+    o2 = orc.run(small)
+    s2 = orc.summarize(small, o2["counters"], o2["hist"], 12, o2["complog"])[0]
+    assert s2["percentile_source"] == 1 and s2["p95_latency"] == 7.0
 
 
 # ---------------------------------------------------------------- Algorithm 1 (per-class budgets, known lengths)

@@ -23,6 +23,7 @@ def _same(a, b):
             assert ga[k] == gb[k], k
         for k in FLOATS:                      # fp64 summaries: relative 1e-9 as everywhere else
             assert abs(ga[k] - gb[k]) <= 1e-9 * max(abs(gb[k]), 1e-300), k
+        assert ga["percentile_source"] == gb["percentile_source"]
 
 
 def test_two_calls_in_a_row_match_fcsim_stats():
