@@ -29,16 +29,15 @@ if ROOT not in sys.path:
 METRIC = "simulated replica-steps/s"
 UNIT = "replica-steps/s"
 
-# Executed warp-instructions per replica-step of the step kernels in the timed regime of each preset, from the
-# committed ncu captures (profiles/): smsp__inst_executed.sum over the launches of one bench step (one kernel per
-# policy present) / (replicas x slots).  None = not captured for the current kernels.
-INST_PER_REPLICA_STEP = {1: 240.8, 2: 261.4, 3: 289.9, 4: 396.4, 5: 195.0, 6: 2016.7}
-# DRAM bytes (read + write) per replica-step from the same captures, None = not captured.
-DRAM_BYTES_PER_REPLICA_STEP = {1: 30.0, 2: 19.7, 3: 21.4, 4: 12.8, 5: 9.3, 6: 38.4}
+# Executed warp-instructions and DRAM bytes per replica-step of the step kernels come from ncu captures and are
+# kept, with the SHA-256 of the kernel sources they were taken on, in profiles/kernel_constants.json
+# (written by paper_2604_11001_b200/profile_constants.py).  When the sources have changed since, the figures that
+# depend on them are printed as null and the line says that the constants are stale.
 
-DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 2000, 6: 500}
+DEFAULT_CHUNK = {1: 200, 2: 1000, 3: 2000, 4: 2000, 5: 4000, 6: 500}
 NAMES = {1: "cfg1-tiny-flow", 2: "cfg2-policy-comparison", 3: "cfg3-stability-sweep", 4: "cfg4-heavy-tail",
          5: "cfg5-large-bursty", 6: "cfg6-paper-section-4.1"}
+SIDE_WORKLOADS = (1, 2, 3, 4, 6)     # reported next to the headline workload in the default run
 
 
 def make_config(workload: int, total_steps: int, rank: int = 0, replicas: int = 0):
@@ -174,46 +173,20 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=5, choices=[1, 2, 3, 4, 5, 6])
-    ap.add_argument("--chunk", type=int, default=0, help="slots per bench step (0 = preset default)")
-    ap.add_argument("--replicas", type=int, default=0, help="replicas per group (0 = the preset's; profiling aid)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 0)
-
-    if args.impl == "reference":
-        run_reference(args)
-        return
-
+def run_workload(args, workload, steps, warmup, chunk, cpu_seconds, ctx):
+    """One workload through the device-buffer path (timed with CUDA events), the host-buffer path (wall clock) and
+    the CPU checker (bounded sample); returns the fields of a bench line."""
     import torch
     from paper_2604_11001_b200 import binding as fb
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-
-    chunk = args.chunk or DEFAULT_CHUNK[args.workload]
-    total_steps = (args.warmup + args.steps) * chunk
-    cfg = make_config(args.workload, total_steps, rank, args.replicas)
+    from paper_2604_11001_b200 import profile_constants as pc
+    rank, world, local_rank, dist = ctx["rank"], ctx["world"], ctx["local_rank"], ctx["dist"]
+    total_steps = (warmup + steps) * chunk
+    cfg = make_config(workload, total_steps, rank, args.replicas)
 
     # CPU baseline first (rank 0 only): no GPU work is in flight while the host cores are timed
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores, desc, dt = sized_oracle_sample(args.workload, 2000 if args.workload == 1 else 3000, 15.0)
+    if rank == 0 and world == 1 and cpu_seconds > 0:
+        v, cores, desc, dt = sized_oracle_sample(workload, 2000 if workload == 1 else 3000, cpu_seconds)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
                         "seconds": round(dt, 2)}
 
@@ -228,24 +201,24 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         sim.run(chunk, stream)
     barrier()
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     ev[0].record(stream)
-    for i in range(args.steps):
+    for i in range(steps):
         sim.run(chunk, stream)
         ev[i + 1].record(stream)
     barrier()
     clocks = sampler.stop() if sampler else None
     ms_total = ev[0].elapsed_time(ev[-1])
-    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     if dist is not None:
         tmax = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         ms_total = float(tmax.item())
-    value = world * R * chunk * args.steps / (ms_total * 1e-3)
+    value = world * R * chunk * steps / (ms_total * 1e-3)
     n_policies = len({g.policy for g in cfg.groups})   # one kernel per policy, side by side on forked streams
     launches_per_step = -(-chunk // info["max_steps_per_launch"]) * n_policies
 
@@ -272,13 +245,14 @@ def main():
         out = fb.fcsim_simulate_host(cfg, total_steps, out=host)
         dt = time.perf_counter() - t0
         assert (out["counters"] == counters).all(), "host-buffer run differs from the device-buffer run"
+        del host, out
         if dist is not None:
             tm = torch.tensor([dt], device="cuda", dtype=torch.float64)
             dist.all_reduce(tm, op=dist.ReduceOp.MAX)
             dt = float(tm.item())
         table_bytes = 4 * (cfg.class_law.n + sum(t.n for t in cfg.prompt) + sum(t.n for t in cfg.decode)
                            + sum(t.n for a in cfg.arrivals for t in a.count))
-        n_all = args.warmup + args.steps
+        n_all = warmup + steps
         e2e = {"value": world * R * total_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": world * table_bytes / n_all,
                "d2h_bytes_per_step": world * (out_bytes + sizes["scratch"]) / n_all,
@@ -287,14 +261,13 @@ def main():
                        % (total_steps, n_all),
                "seconds": round(dt, 3)}
 
-    if rank != 0:
-        dist.destroy_process_group()
-        return
     peaks, peak_kind = measured_peaks()
     sm_mhz = (clocks or {}).get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
     peak_ginst = info["sm_count"] * 4 * sm_mhz * 1e6 / 1e9       # warp-instructions/s the schedulers can issue
-    ipr = INST_PER_REPLICA_STEP.get(args.workload)
-    dbr = DRAM_BYTES_PER_REPLICA_STEP.get(args.workload)
+    consts = pc.load()
+    k = None if (consts["stale"] or args.replicas) else consts["presets"].get(str(workload))
+    ipr = k["inst_per_replica_step"] if k else None
+    dbr = k["dram_bytes_per_replica_step"] if k else None
     kernel_ms = statistics.mean(per_step) / (launches_per_step // n_policies)
     roofline = {
         "bound": "alu",
@@ -305,6 +278,11 @@ def main():
         "frac": (ipr * value / world / 1e9 / peak_ginst) if ipr else None,
         "traffic": (dbr * R * min(chunk, info["max_steps_per_launch"])) if dbr else None,
         "inst_per_replica_step": ipr,
+        "ncu_issue_active_pct": [round(x["issue_active_pct"], 1) for x in k["kernels"]] if k else None,
+        "constants": {"file": "profiles/kernel_constants.json", "sha256_at_capture": consts.get("sha256"),
+                      "sha256_now": pc.source_hash(), "stale": bool(consts["stale"]),
+                      "captured_on": ({"replicas": k["replicas"], "slots": k["slots"]} if k else None)},
+        "constants_stale": bool(consts["stale"]),
         "peak_basis": "%d SMs x 4 schedulers x %.0f MHz (median SM clock sampled during the timed region)"
                       % (info["sm_count"], sm_mhz),
         "kernel_ms_per_launch": kernel_ms, "launches_per_step": launches_per_step, "policies": n_policies,
@@ -314,12 +292,10 @@ def main():
         rec_bytes = 8.0 / cfg.trace_stride
         roofline["trace_stream_gbs"] = value / world * rec_bytes / 1e9
         roofline["trace_stream_frac_of_hbm"] = roofline["trace_stream_gbs"] / peaks.get("hbm_gbs", 6650.0)
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": NAMES[args.workload], "replicas_per_gpu": R, "slots_per_step": chunk,
-                   "warm_slots": args.warmup * chunk, "groups": len(cfg.groups), "M": cfg.M, "K": cfg.K,
+    return {
+        "value": value, "ms_per_step": ms_total / steps, "steps": steps, "warmup": warmup,
+        "config": {"workload": NAMES[workload], "replicas_per_gpu": R, "slots_per_step": chunk,
+                   "warm_slots": warmup * chunk, "groups": len(cfg.groups), "M": cfg.M, "K": cfg.K,
                    "Qcap": cfg.Qcap, "Acap": cfg.Acap,
                    "l2": ("replica state %.0f MB exceeds the 126 MB L2; no explicit flush" % (sizes["workspace"] / 1e6)
                           if sizes["workspace"] > 126e6 else
@@ -327,11 +303,86 @@ def main():
                           "not; no explicit flush" % (sizes["workspace"] / 1e6,
                                                      (sizes["trace"] + sizes["complog"] + sizes["hist"]) / 1e6)),
                    "launch": info, "parallelism": "replicas only, %d per GPU" % R},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_step,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": steps * launches_per_step,
         "roofline": roofline, "cpu_baseline": cpu_baseline,
         "check": {"replica_steps_done": done_steps, "completed": int(counters[:, 5].sum()),
-                  "mean_latency": [round(s["mean_latency"], 3) for s in summary[:4]]},
+                  "mean_latency": [round(s["mean_latency"], 3) for s in summary[:4]],
+                  "p95_latency": [s["p95_latency"] for s in summary[:4]],
+                  "percentile_source": [s["percentile_source"] for s in summary[:4]]},
     }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=5, choices=[1, 2, 3, 4, 5, 6])
+    ap.add_argument("--chunk", type=int, default=0, help="slots per bench step (0 = preset default)")
+    ap.add_argument("--replicas", type=int, default=0, help="replicas per group (0 = the preset's; profiling aid)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-side-workloads", action="store_true",
+                    help="only the headline workload (the default run also reports the other presets)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    ctx = {"rank": rank, "world": world, "local_rank": local_rank, "dist": dist}
+
+    chunk = args.chunk or DEFAULT_CHUNK[args.workload]
+    if args.workload == 5 and not args.chunk:
+        # the horizon of the large bursty run is 100 000 slots: with the default 5 + 20 steps the run is exactly that
+        chunk = min(chunk, max(1, 100000 // max(1, args.warmup + args.steps)))
+    head = run_workload(args, args.workload, args.steps, args.warmup, chunk,
+                        0.0 if args.no_cpu_baseline else 15.0, ctx)
+
+    # the other presets, three timed steps each after five warm-up steps (1 GPU, headline workload only)
+    side = None
+    if args.workload == 5 and world == 1 and not args.no_side_workloads and not args.replicas:
+        side = {}
+        for w in SIDE_WORKLOADS:
+            r = run_workload(args, w, 3, 5, DEFAULT_CHUNK[w], 0.0 if args.no_cpu_baseline else 5.0, ctx)
+            rf = r["roofline"]
+            side[NAMES[w]] = {
+                "value": r["value"], "unit": UNIT, "ms_per_step": r["ms_per_step"], "steps": 3, "warmup": 5,
+                "slots_per_step": DEFAULT_CHUNK[w], "replicas": r["config"]["replicas_per_gpu"],
+                "frac": rf["frac"], "inst_per_replica_step": rf["inst_per_replica_step"],
+                "ncu_issue_active_pct": rf["ncu_issue_active_pct"], "constants_stale": rf["constants_stale"],
+                "trace_stream_gbs": rf.get("trace_stream_gbs"),
+                "trace_stream_frac_of_hbm": rf.get("trace_stream_frac_of_hbm"),
+                "e2e": r["e2e"], "cpu_baseline": r["cpu_baseline"], "clocks": r["clocks"],
+                "gpu_launches": r["gpu_launches"], "check": r["check"]}
+
+    if rank != 0:
+        dist.destroy_process_group()
+        return
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": head["config"], "clocks": head["clocks"], "e2e": head["e2e"],
+        "gpu_launches": head["gpu_launches"], "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"],
+        "check": head["check"],
+    }
+    if side is not None:
+        line["workloads"] = side
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
