@@ -70,6 +70,14 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def wait_first_sample(self, timeout_s: float = 3.0):
+        """Block until nvidia-smi has written its first line (its start-up takes longer than a short timed region)."""
+        t0 = time.perf_counter()
+        while self.proc is not None and time.perf_counter() - t0 < timeout_s:
+            if os.path.getsize(self.tmp.name) > 0:
+                return
+            time.sleep(0.02)
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
@@ -201,17 +209,32 @@ def run_workload(args, workload, steps, warmup, chunk, cpu_seconds, ctx):
             dist.barrier()
             torch.cuda.synchronize()
 
+    # Clock record: sampled during the timed region.  A workload whose whole run is shorter than the sampler's
+    # period (presets 1 and 2: milliseconds) is sampled over warm-up and timed steps together, repeated until the
+    # window holds samples, and the record says so.
+    est_ms = R * chunk * steps / 3.0e6          # at about 3e9 replica-steps/s
+    short = est_ms < 400.0
+    sampler = None
+    if rank == 0 and short:
+        sampler = ClockSampler(local_rank)
+        sampler.wait_first_sample()
     for _ in range(warmup):
         sim.run(chunk, stream)
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if rank == 0 and not short:
+        sampler = ClockSampler(local_rank)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     ev[0].record(stream)
     for i in range(steps):
         sim.run(chunk, stream)
         ev[i + 1].record(stream)
     barrier()
+    if sampler is not None and short:
+        time.sleep(0.25)                        # at least two sampler periods inside the window
     clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["window"] = ("warm-up and timed steps plus 0.25 s (the run is shorter than the sampler's period)"
+                            if short else "timed steps")
     ms_total = ev[0].elapsed_time(ev[-1])
     per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     if dist is not None:

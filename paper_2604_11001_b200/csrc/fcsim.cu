@@ -33,6 +33,7 @@ struct Layout {
     size_t tstage_off;                          // trace staging buffers, 0 = unused
     size_t state_bytes;                         // ring + state words (+ projection words) saved between launches
     int has_v;
+    uint32_t prof_mask;                         // MC benchmark: H - 1 when the projection is kept per future slot, else 0
     int warps_per_block;
     int n_rec;
     long long R;
@@ -123,9 +124,20 @@ int plan(const fcsim_config* c, Layout* L) {
     while ((long long)L->QC < rc) L->QC <<= 1;
     L->Apad = (int)align_up((size_t)c->Acap, 4);
     L->S = (int)align_up((size_t)std::max(128, max_count), 2);
-    // the MC benchmark keeps one more word per active entry (projected usage in its last slot), saved with the state
-    L->state_bytes = (size_t)L->Apad * 8 + (size_t)L->Apad * 4 * (any_mc ? 2 : 1);
+    // The MC benchmark keeps its projection of the future memory usage with the state: one word per active entry
+    // (usage in that request's last slot), or, when that is no larger, one word per future slot (a ring of H slots,
+    // H the power of two above the longest output length): a test then walks the candidate's lifetime instead of
+    // the active set.
     L->has_v = any_mc ? 1 : 0;
+    L->prof_mask = 0;
+    size_t proj_words = 0;
+    if (any_mc) {
+        uint32_t H = 32;
+        while ((int64_t)H < omax + 1) H <<= 1;
+        if ((int64_t)H <= (int64_t)L->Apad) L->prof_mask = H - 1;
+        proj_words = L->prof_mask ? H : (size_t)L->Apad;
+    }
+    L->state_bytes = (size_t)L->Apad * 8 + (size_t)L->Apad * 4 + proj_words * 4;
     // workspace record of a replica: 16 header words, the saved shared-memory state, the queue ring
     L->gq_off = kHeaderWords * 4 + L->state_bytes;
     L->ws_stride = L->gq_off + (size_t)L->QC * 8;
@@ -435,6 +447,7 @@ static step_kernel_t pick_step_kernel(int policy, int ctas, int rec) {
         case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec);
         case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec);
         case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec);
+        case 6: return step_kernel_for<6>(ctas, rec);  // the MC benchmark with its projection per future slot
         default: return nullptr;
     }
 }
@@ -734,7 +747,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
                 block += tab_extra;
             }
             for (int ctas = 5; ctas <= 7; ++ctas) {
-                step_kernel_t k = pick_step_kernel(pl.policy, ctas, rec);
+                step_kernel_t k = pick_step_kernel(pl.policy == FCSIM_POLICY_MC && L.prof_mask ? 6 : pl.policy, ctas, rec);
                 if (!k) return fail(FCSIM_EINVAL);
                 int occ = 0;
                 {
@@ -801,6 +814,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.tstage_off = (uint32_t)L.tstage_off;
     p.state_bytes = (uint32_t)L.state_bytes;
     p.has_v = L.has_v;
+    p.prof_mask = L.prof_mask;
     p.pool = h->d_pool; p.tables = h->d_tables; p.arrivals = h->d_arrivals;
     p.groups = h->d_pgroups;  // narrowed to the policy's piece at every launch
     p.workspace = static_cast<unsigned char*>(b->workspace);

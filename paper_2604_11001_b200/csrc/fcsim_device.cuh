@@ -13,7 +13,10 @@
 //                      far; 0x40000000 | slot of completion for a request that has completed but whose entry
 //                      has not been squeezed out yet (completed entries are removed lazily, many at a time,
 //                      and their latency statistics are taken then, one entry per lane).
-//   vproj [Acap] i32   only with MC groups: projected memory usage of the last slot of each active entry.
+//   vproj [Acap] i32   only with MC groups, entry form: projected memory usage of the last slot of each active entry.
+//   uprof [H]    i32   only with MC groups, profile form (used when H <= Acap, H the power of two above the longest
+//                      output length): projected memory usage of the future slots, a ring indexed by slot & (H - 1);
+//                      takes the place of vproj.
 //   queue [QC]   u64   the FIFO waiting queue, a ring in the replica's record in GLOBAL memory (QC a power of
 //                      two >= Qcap + Acap: evictions may push the queue past Qcap).  It is touched at its ends
 //                      only: arrivals are appended (plain stores, nobody waits for them), the head is read
@@ -94,7 +97,9 @@ struct Params {
     uint32_t qwin_off;            // byte offset of the queue window in a warp's shared memory
     uint32_t tabcache_off;        // byte offset in the CTA's shared memory of a copy of `tables` (0 = none)
     uint32_t state_bytes;         // ring + state words (+ projection words): what is saved between launches
-    int32_t has_v;                // 1 = a projection word per active entry follows the state words (MC benchmark)
+    int32_t has_v;                // 1 = the MC benchmark's projection words follow the state words
+    uint32_t prof_mask;           // MC benchmark: 0 = one projection word per active entry; else H - 1, the words are
+                                  // the projected usage of the future slots (ring of H slots)
     uint32_t tstage_off;          // byte offset of the trace staging area (2 x 32 records) in a warp's shared
                                   // memory; 0 = records are kept in registers and stored with plain stores
     const DevTable* tables;       // [0] class law, [1 .. nc] prompt, [1+nc .. 2nc] decode
@@ -273,16 +278,19 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 // parameters say (decided at run time).
 // kExt (= kPol >= 4): the per-class activation of Algorithm 1 (policy 4) and the future-memory test of the MC
 // benchmark (policy 5) use extra per-warp state (class counts, projection words).
+// kPol 6 is the MC benchmark again, with its projection kept per future slot instead of per active entry
+// (the host picks it when the longest output length is short next to the active set's storage).
 // kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80).  The host
 // asks the occupancy calculator about both.
 template <int kPol, int kMinCtas, int kRec>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     constexpr bool kExt = kPol >= 4;
+    constexpr bool kMcProfile = kPol == 6;  // MC benchmark, projection per future slot
     // Completed entries tolerated inside the active range before they are squeezed out (they always are when the
     // storage runs out).  The whole-prompt policies touch the range only where a request finishes, so removal
     // as late as possible measured fastest; the policies that walk the range (chunked prefills, Algorithm 1's
     // storage check, the MC projections) want it short.
-    constexpr int kCompactAt = (kPol <= 1 || kPol == 3) ? 256 : 32;
+    constexpr int kCompactAt = (kPol <= 1 || kPol == 3 || kPol == 6) ? 256 : 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // the table descriptors of the length laws are read for every generated arrival: the host reserves room
     // for a copy behind the warps' slices when that does not cost a resident CTA
@@ -476,12 +484,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     acc_w += (unsigned long long)l * o + (unsigned long long)o * (o + 1) / 2;
                     if (hrow) atomicAdd(&HROW(min(lat >> p.hist_shift, p.hist_bins - 1)), 1);
                 }
-                if (kExt && p.has_v && mv) v = vproj[WA(shead + i)];
+                if (kPol == 5 && mv) v = vproj[WA(shead + i)];
                 __syncwarp();
                 if (mv) {
                     RING(WA(shead + i + sh)) = e;
                     STATE(WA(shead + i + sh)) = sw;
-                    if (kExt && p.has_v) vproj[WA(shead + i + sh)] = v;
+                    if (kPol == 5) vproj[WA(shead + i + sh)] = v;
                 }
                 __syncwarp();
                 holes += __popc(m);
@@ -740,7 +748,28 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             gate_closed = (a == 0) && (policy <= 1 || policy == 3);
                             break;
                         }
-                        if (kExt && policy == 5) {
+                        if (kMcProfile) {
+                            // MC benchmark (Section 4.1): start the queue head only if the usage of every future
+                            // slot stays within M.  uprof[tau & mask] is the usage of slot tau >= t if nothing else
+                            // starts; the head would hold l + (tau - t + 1) = a_h + tau in the slots t .. f_h.
+                            // Lane = future slot: one read-only pass tests, a second one books the head.
+                            const uint64_t eh = q_e;
+                            const int op_h = grp.mc_worst != 0 ? (tabs[1 + p.n_classes + entry_cls(eh)].vmin +
+                                                                  (int)tabs[1 + p.n_classes + entry_cls(eh)].n - 1)
+                                                               : entry_o(eh);
+                            const int a_h = l - t + 1;
+                            bool over = false;
+                            for (int base = 0; base < op_h; base += 32) {
+                                const int tau = t + base + lane;
+                                over |= (base + lane < op_h) && (vproj[(uint32_t)tau & p.prof_mask] + a_h + tau > M);
+                            }
+                            if (__any_sync(FULL, over)) { CADD(C_GATE_BLOCKED, 1); break; }
+                            for (int base = 0; base < op_h; base += 32) {
+                                const int tau = t + base + lane;
+                                if (base + lane < op_h) vproj[(uint32_t)tau & p.prof_mask] += a_h + tau;
+                            }
+                        }
+                        if (kPol == 5) {
                             // MC benchmark (Section 4.1): start the queue head only if the usage of every future
                             // slot stays within M.  With a_i = l_i - (activation slot) + 1, request i holds a_i + tau
                             // in slot tau up to its last slot f_i; the usage can only peak in some last slot.
@@ -1002,7 +1031,25 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     STATE(WA(shead + i)) = kDead | (uint32_t)t;
                                 }
                                 ndone += __popc(m);
-                                if (kExt && policy == 5 && grp.mc_worst != 0) {
+                                if (kMcProfile && grp.mc_worst != 0) {
+                                    // worst-case projection: a request that ends before its projected last slot
+                                    // f_c = t + (longest output of its class - o) leaves the projected usage of the
+                                    // slots t+1 .. f_c, where it was booked with a_c + tau, a_c = l + o - t
+                                    uint32_t mm = m;
+                                    while (mm) {
+                                        const int src = __ffs(mm) - 1;
+                                        mm &= mm - 1;
+                                        const uint64_t ec = __shfl_sync(FULL, e, src);
+                                        const DevTable dc = tabs[1 + p.n_classes + entry_cls(ec)];
+                                        const int extra = dc.vmin + (int)dc.n - 1 - entry_o(ec);  // slots it leaves early
+                                        const int a_c = entry_l(ec) + entry_o(ec) - t;
+                                        for (int base = 0; base < extra; base += 32) {
+                                            const int tau = t + 1 + base + lane;
+                                            if (base + lane < extra) vproj[(uint32_t)tau & p.prof_mask] -= a_c + tau;
+                                        }
+                                    }
+                                }
+                                if (kPol == 5 && grp.mc_worst != 0) {
                                     // MC benchmark with worst-case projection: a request that ends before its
                                     // projected last slot f_c leaves the projected usage of every last slot <= f_c.
                                     // The slot's early finishers are collected, one per lane, and taken out of the
@@ -1025,7 +1072,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         }
                         if (lane == c) cmin = gmin;
                     }
-                    if (kExt && npend > 0) mc_release();
+                    if (kPol == 5 && npend > 0) mc_release();
                     next_fin = __reduce_min_sync(FULL, cmin);
                     if (ndone > 0) {
                         gate_closed = false;
@@ -1039,6 +1086,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         }
                         __syncwarp();
                     }
+                }
+
+                if (kMcProfile) {  // slot t has passed: its place in the ring is slot t + H's, which nothing reaches yet
+                    __syncwarp();
+                    if (lane == 0) vproj[(uint32_t)t & p.prof_mask] = 0;
                 }
 
                 // ---- record
