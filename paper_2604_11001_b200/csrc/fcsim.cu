@@ -65,6 +65,36 @@ bool table_ok(const fcsim_table& t, int64_t vmin_lo, int64_t vmax_hi) {
     return true;
 }
 
+// First and second moment of the law a table realises (value vmin + k has the mass between thresholds k - 1 and k,
+// the last value the rest).
+void table_moments(const fcsim_table& t, double* m1, double* m2) {
+    double prev = 0.0, a = 0.0, b = 0.0;
+    for (uint32_t k = 0; k < t.n; ++k) {
+        const double cum = k + 1 < t.n ? std::max(prev, (double)t.cdf[k] / 4294967296.0) : 1.0;
+        const double v = (double)t.vmin + k;
+        a += v * (cum - prev);
+        b += v * v * (cum - prev);
+        prev = cum;
+    }
+    *m1 = a;
+    if (m2) *m2 = b;
+}
+
+// Requests per slot that the cache can serve in the long run: M / E[w], with the per-request workload
+// w = l o + o (o + 1) / 2 of Prop. 3.5 (l and o independent within a class).
+double capacity_rate(const fcsim_config* c) {
+    double ew = 0.0, prev = 0.0;
+    for (int k = 0; k < c->n_classes; ++k) {
+        const double cum = k + 1 < c->n_classes ? std::max(prev, (double)c->class_law.cdf[k] / 4294967296.0) : 1.0;
+        double el, eo, eo2;
+        table_moments(c->prompt[k], &el, nullptr);
+        table_moments(c->decode[k], &eo, &eo2);
+        ew += (cum - prev) * (el * eo + 0.5 * (eo + eo2));
+        prev = cum;
+    }
+    return ew > 0.0 ? (double)c->M / ew : 0.0;
+}
+
 // Validates the description and derives the storage layout.  Returns an FCSIM_* code.
 int plan(const fcsim_config* c, Layout* L) {
     if (!c) return FCSIM_EINVAL;
@@ -421,33 +451,40 @@ typedef void (*step_kernel_t)(const Params);
 // not change it between another handle's two steps.
 static std::mutex g_kernel_attr_mutex;
 
-// The step kernel compiled for one policy, for a register allocation that lets 6 or 5 CTAs reside on an SM, and
-// for what is recorded per slot (0 nothing, 1 trace only, 2 decided at run time; Algorithm 1 and the MC benchmark
-// exist in the run-time form only).
+// The step kernel compiled for one policy, for a register allocation that lets 7, 6 or 5 CTAs reside on an SM, for
+// what is recorded per slot (0 nothing, 1 trace only, 2 decided at run time; Algorithm 1 and the MC benchmark
+// exist in the run-time form only) and, for the whole-prompt first-come-first-served policies, with or without the
+// activation of several queue heads at once.
 template <int kPol, int kCtas>
-static step_kernel_t step_kernel_for(int rec) {
-    if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2>;
-    constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 and 5 uninstantiated
-    if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1>;
-    return fcsim_step_kernel<kP, kCtas, 0>;
+static step_kernel_t step_kernel_for(int rec, bool bulk) {
+    constexpr bool kFifo = kPol <= 1 || kPol == 3;
+    constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 .. 6 uninstantiated
+    if (kFifo && bulk) {
+        if (rec == 2) return fcsim_step_kernel<kP, kCtas, 2, kFifo>;
+        if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, kFifo>;
+        return fcsim_step_kernel<kP, kCtas, 0, kFifo>;
+    }
+    if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, false>;
+    if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, false>;
+    return fcsim_step_kernel<kP, kCtas, 0, false>;
 }
 template <int kPol>
-static step_kernel_t step_kernel_for(int ctas, int rec) {
+static step_kernel_t step_kernel_for(int ctas, int rec, bool bulk) {
     switch (ctas) {
-        case 5: return step_kernel_for<kPol, 5>(rec);
-        case 6: return step_kernel_for<kPol, 6>(rec);
-        default: return step_kernel_for<kPol, 7>(rec);
+        case 5: return step_kernel_for<kPol, 5>(rec, bulk);
+        case 6: return step_kernel_for<kPol, 6>(rec, bulk);
+        default: return step_kernel_for<kPol, 7>(rec, bulk);
     }
 }
-static step_kernel_t pick_step_kernel(int policy, int ctas, int rec) {
+static step_kernel_t pick_step_kernel(int policy, int ctas, int rec, bool bulk) {
     switch (policy) {
-        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(ctas, rec);
-        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(ctas, rec);
-        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(ctas, rec);
-        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec);
-        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec);
-        case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec);
-        case 6: return step_kernel_for<6>(ctas, rec);  // the MC benchmark with its projection per future slot
+        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(ctas, rec, bulk);
+        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(ctas, rec, bulk);
+        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(ctas, rec, bulk);
+        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec, bulk);
+        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec, bulk);
+        case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec, bulk);
+        case 6: return step_kernel_for<6>(ctas, rec, bulk);  // the MC benchmark with its projection per future slot
         default: return nullptr;
     }
 }
@@ -459,6 +496,7 @@ struct PolicyLaunch {
     step_kernel_t kernel = nullptr;
     int pg_off = 0, pg_cnt = 0;   // its groups in d_pgroups
     int n_work = 0;               // replicas
+    bool bulk = false;            // two or more requests arrive, and may be activated, per slot on average
     int warps_per_block = 0, blocks_per_sm = 0, grid = 0;
     size_t smem_block = 0, tabcache_off = 0;
     cudaStream_t side = nullptr;  // null: the caller's stream
@@ -617,17 +655,30 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
     }
     // the same groups sorted by policy (order within a policy kept): one launch per policy walks its piece
     std::vector<DevGroup> pgrps;
+    const double cap_rate = capacity_rate(c);
     for (int pol = FCSIM_POLICY_MC; pol >= FCSIM_POLICY_FLOW; --pol) {  // costly policies first
         PolicyLaunch pl;
         pl.policy = pol;
         pl.pg_off = (int)pgrps.size();
+        double most = 0.0;  // requests that arrive and may be activated per slot, the largest over the policy's groups
         for (int g = 0; g < c->n_groups; ++g) {
             if (grps[g].policy != pol) continue;
             DevGroup d = grps[g];
             d.wfirst = pl.n_work;
             pl.n_work += d.n;
             pgrps.push_back(d);
+            const fcsim_arrivals& A = c->arrivals[d.arrivals_id];
+            double rate = 0.0;
+            for (uint32_t st = 0; st < A.n_states; ++st) {
+                double m;
+                table_moments(A.count[st], &m, nullptr);
+                rate = std::max(rate, m);
+            }
+            if (pol == FCSIM_POLICY_FLOW) rate = std::min(rate, (double)d.b_fp / 65536.0);
+            most = std::max(most, rate);
         }
+        // activations per slot cannot outrun the arrivals, the flow-control rate or what the cache can serve
+        pl.bulk = std::min(most, cap_rate) >= 2.0;
         pl.pg_cnt = (int)pgrps.size() - pl.pg_off;
         if (pl.pg_cnt > 0) h->launches.push_back(pl);
     }
@@ -672,7 +723,9 @@ static void release(fcsim* h) {
     delete h;
 }
 
-extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_t** out) {
+// trace_window_recs: 0 = the trace buffer holds the whole horizon ([R][T_max / stride] records); otherwise it is a
+// window of that many records per replica which the caller of launch_slots moves along the horizon.
+static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_t** out, int trace_window_recs) {
     if (!out) return FCSIM_EINVAL;
     *out = nullptr;
     Layout L;
@@ -681,6 +734,7 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     if (!b) return FCSIM_ESIZE;
     fcsim_sizes sz;
     sizes_of(cfg, L, &sz);
+    if (trace_window_recs > 0) sz.trace = (size_t)L.R * (size_t)trace_window_recs * 8;
     if (!b->workspace || !b->counters || !b->scratch) return FCSIM_ESIZE;
     if (sz.trace && !b->trace) return FCSIM_ESIZE;
     if (sz.hist && !b->hist) return FCSIM_ESIZE;
@@ -747,7 +801,8 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
                 block += tab_extra;
             }
             for (int ctas = 5; ctas <= 7; ++ctas) {
-                step_kernel_t k = pick_step_kernel(pl.policy == FCSIM_POLICY_MC && L.prof_mask ? 6 : pl.policy, ctas, rec);
+                step_kernel_t k = pick_step_kernel(pl.policy == FCSIM_POLICY_MC && L.prof_mask ? 6 : pl.policy, ctas, rec,
+                                                   pl.bulk);
                 if (!k) return fail(FCSIM_EINVAL);
                 int occ = 0;
                 {
@@ -806,7 +861,8 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
     p.key0 = (uint32_t)(cfg->seed & 0xffffffffu);
     p.key1 = (uint32_t)(cfg->seed >> 32);
     p.n_classes = cfg->n_classes; p.n_groups = cfg->n_groups; p.n_replicas = (int)L.R;
-    p.trace_stride = cfg->trace_stride; p.n_rec = L.n_rec;
+    p.trace_stride = cfg->trace_stride; p.n_rec = trace_window_recs > 0 ? trace_window_recs : L.n_rec;
+    p.rec_base = 0;
     p.hist_bins = cfg->hist_bins; p.hist_shift = cfg->hist_shift; p.complog_cap = cfg->complog_cap;
     p.gpool = h->d_gpool;
     p.bclass = h->d_bclass;
@@ -839,12 +895,46 @@ extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcs
 //                                                                 requests running at its start already held)
 // so n <= (2^32 - 2^30 - 1) / (Qcap + 2 Acap) keeps all of them exact (M <= 2^30); with Qcap + Acap <= 2^20 that
 // is at least 1536 slots.
+extern "C" int fcsim_create(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_t** out) {
+    return create_handle(cfg, b, out, 0);
+}
+
 static int max_steps_per_launch(const fcsim* h) {
     long long s = kTargetWorkPerLaunch / std::max<long long>(1, h->L.R);
     s = std::max<long long>(256, std::min<long long>(s, kMaxStepsPerLaunch));
     const long long per_slot = (long long)h->cfg.Qcap + 2LL * h->cfg.Acap;
     s = std::min<long long>(s, ((1LL << 32) - (1LL << 30) - 1) / per_slot);
     return (int)std::max<long long>(1, s);
+}
+
+// One group of concurrent launches (one kernel per policy present) advancing every replica by `now` slots.
+static int launch_slots(fcsim* h, int now, cudaStream_t st) {
+    CUDA_TRY(h, cudaMemsetAsync(h->d_work, 0, 8 * sizeof(unsigned int), st));  // one work counter per policy
+    if (h->launches.size() > 1) CUDA_TRY(h, cudaEventRecord(h->fork, st));
+    for (const PolicyLaunch& pl : h->launches) {
+        cudaStream_t ls = pl.side ? pl.side : st;
+        if (pl.side) CUDA_TRY(h, cudaStreamWaitEvent(pl.side, h->fork, 0));
+        Params p = h->params;
+        p.t0 = h->t_done;
+        p.n_steps = now;
+        p.groups = h->d_pgroups + pl.pg_off;
+        p.n_groups = pl.pg_cnt;
+        p.n_work = pl.n_work;
+        p.work_counter = h->d_work + pl.policy;
+        p.tabcache_off = (uint32_t)pl.tabcache_off;
+        {
+            // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
+            std::lock_guard<std::mutex> lock(g_kernel_attr_mutex);
+            CUDA_TRY(h, cudaFuncSetAttribute(pl.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_block));
+            pl.kernel<<<pl.grid, pl.warps_per_block * 32, pl.smem_block, ls>>>(p);
+            CUDA_TRY(h, cudaGetLastError());
+        }
+        if (pl.side) CUDA_TRY(h, cudaEventRecord(pl.done, pl.side));
+    }
+    for (const PolicyLaunch& pl : h->launches)
+        if (pl.side) CUDA_TRY(h, cudaStreamWaitEvent(st, pl.done, 0));
+    h->t_done += now;
+    return FCSIM_OK;
 }
 
 extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
@@ -856,31 +946,7 @@ extern "C" int fcsim_run(fcsim_t* h, int32_t n_steps, void* cuda_stream) {
     int left = n_steps;
     while (left > 0) {
         const int now = std::min(left, per);
-        CUDA_TRY(h, cudaMemsetAsync(h->d_work, 0, 8 * sizeof(unsigned int), st));  // one work counter per policy
-        if (h->launches.size() > 1) CUDA_TRY(h, cudaEventRecord(h->fork, st));
-        for (const PolicyLaunch& pl : h->launches) {
-            cudaStream_t ls = pl.side ? pl.side : st;
-            if (pl.side) CUDA_TRY(h, cudaStreamWaitEvent(pl.side, h->fork, 0));
-            Params p = h->params;
-            p.t0 = h->t_done;
-            p.n_steps = now;
-            p.groups = h->d_pgroups + pl.pg_off;
-            p.n_groups = pl.pg_cnt;
-            p.n_work = pl.n_work;
-            p.work_counter = h->d_work + pl.policy;
-            p.tabcache_off = (uint32_t)pl.tabcache_off;
-            {
-                // the limit is a property of the kernel, not of the handle: another handle may have lowered it since
-                std::lock_guard<std::mutex> lock(g_kernel_attr_mutex);
-                CUDA_TRY(h, cudaFuncSetAttribute(pl.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_block));
-                pl.kernel<<<pl.grid, pl.warps_per_block * 32, pl.smem_block, ls>>>(p);
-                CUDA_TRY(h, cudaGetLastError());
-            }
-            if (pl.side) CUDA_TRY(h, cudaEventRecord(pl.done, pl.side));
-        }
-        for (const PolicyLaunch& pl : h->launches)
-            if (pl.side) CUDA_TRY(h, cudaStreamWaitEvent(st, pl.done, 0));
-        h->t_done += now;
+        if (int rc = launch_slots(h, now, st)) return rc;
         left -= now;
     }
     return FCSIM_OK;
@@ -1089,18 +1155,48 @@ extern "C" const char* fcsim_strerror(int code) {
     }
 }
 
+// Whole job with host buffers.  A large trace does not wait for the end of the run: the device holds two
+// windows of the horizon (a few thousand records per replica each); while the kernels fill one, the other, already
+// full, travels to the caller's rows with one strided copy on a second stream.  The rest of the outputs (counters,
+// histograms, completion log) is copied after the last slot.
 extern "C" int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcsim_counters* host_counters,
                                    void* host_trace, void* host_hist, void* host_complog,
                                    fcsim_summary* per_group_out) {
     fcsim_sizes sz;
     int rc = fcsim_query_sizes(cfg, &sz);
     if (rc != FCSIM_OK) return rc;
+    if (n_steps < 0 || n_steps > cfg->T_max) return FCSIM_ERANGE;
+    Layout L;
+    plan(cfg, &L);
+    // Streaming pays when the trace is large and a replica's piece of a window is long enough for the strided
+    // copy to run at full speed (16 KB and more; rows of a few KB copy at a fraction of it).
+    const long long stride = cfg->trace_stride;
+    const long long recs_run = stride > 0 ? n_steps / stride : 0;
+    long long win_recs = 0;
+    if (host_trace && sz.trace >= ((size_t)256 << 20) && recs_run >= 3 * 2048) {
+        win_recs = std::max<long long>(2048, (((long long)64 << 20) / (L.R * 8) + 31) / 32 * 32);
+        // a window is filled by whole launches
+        const long long per_launch = ((1LL << 31) / std::max<long long>(1, L.R)) / (32 * stride) * 32;
+        win_recs = std::min(win_recs, std::max<long long>(0, per_launch));
+        if (win_recs < 2048 || win_recs * 3 > recs_run) win_recs = 0;
+    }
     fcsim_buffers b;
     std::memset(&b, 0, sizeof(b));
     void** slots[6] = {&b.workspace, &b.counters, &b.trace, &b.hist, &b.complog, &b.scratch};
-    const size_t bytes[6] = {sz.workspace, sz.counters, sz.trace, sz.hist, sz.complog, sz.scratch};
+    size_t bytes[6] = {sz.workspace, sz.counters, sz.trace, sz.hist, sz.complog, sz.scratch};
+    if (win_recs > 0) bytes[2] = 2 * (size_t)L.R * (size_t)win_recs * 8;
+    cudaStream_t run_st = nullptr, copy_st = nullptr;
+    cudaEvent_t filled[2] = {nullptr, nullptr}, sent[2] = {nullptr, nullptr};
+    fcsim_t* h = nullptr;
     auto free_all = [&]() {
+        if (h) fcsim_destroy(h);
         for (void** s : slots) cudaFree(*s);
+        for (int i = 0; i < 2; ++i) {
+            if (filled[i]) cudaEventDestroy(filled[i]);
+            if (sent[i]) cudaEventDestroy(sent[i]);
+        }
+        if (run_st) cudaStreamDestroy(run_st);
+        if (copy_st) cudaStreamDestroy(copy_st);
     };
     for (int i = 0; i < 6; ++i) {
         if (bytes[i] && cudaMalloc(slots[i], bytes[i]) != cudaSuccess) {
@@ -1108,19 +1204,67 @@ extern "C" int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcs
             return FCSIM_ECUDA;
         }
     }
-    fcsim_t* h = nullptr;
-    rc = fcsim_create(cfg, &b, &h);
-    if (rc == FCSIM_OK) rc = fcsim_run(h, n_steps, nullptr);
-    if (rc == FCSIM_OK) rc = fcsim_stats(h, nullptr, host_counters, per_group_out);
+    rc = create_handle(cfg, &b, &h, (int)win_recs);
+    if (rc != FCSIM_OK) { free_all(); return rc; }
+    if (win_recs == 0) {
+        rc = fcsim_run(h, n_steps, nullptr);
+    } else {
+        cudaError_t e = cudaStreamCreateWithFlags(&run_st, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&copy_st, cudaStreamNonBlocking);
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&filled[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sent[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) { free_all(); return FCSIM_ECUDA; }
+        const size_t win_bytes = (size_t)L.R * (size_t)win_recs * 8;
+        const size_t row_bytes = (size_t)L.n_rec * 8;  // the caller's rows hold the whole horizon
+        const int per = max_steps_per_launch(h);
+        long long rec0 = 0;
+        for (int piece = 0; rc == FCSIM_OK && h->t_done < n_steps; ++piece) {
+            const int buf = piece & 1;
+            const long long slots_now = std::min<long long>(win_recs * stride, (long long)n_steps - h->t_done);
+            const long long recs_now = (h->t_done + slots_now) / stride - rec0;
+            unsigned char* win = static_cast<unsigned char*>(b.trace) + (size_t)buf * win_bytes;
+            if (piece >= 2 && cudaStreamWaitEvent(run_st, sent[buf], 0) != cudaSuccess) { rc = FCSIM_ECUDA; break; }
+            h->params.trace = reinterpret_cast<int2*>(win);
+            h->params.rec_base = (int32_t)rec0;
+            long long left = slots_now;
+            while (rc == FCSIM_OK && left > 0) {
+                const int now = (int)std::min<long long>(left, per);
+                rc = launch_slots(h, now, run_st);
+                left -= now;
+            }
+            if (rc != FCSIM_OK) break;
+            e = cudaEventRecord(filled[buf], run_st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(copy_st, filled[buf], 0);
+            if (e == cudaSuccess && recs_now > 0)
+                e = cudaMemcpy2DAsync(static_cast<unsigned char*>(host_trace) + (size_t)rec0 * 8, row_bytes, win,
+                                      (size_t)win_recs * 8, (size_t)recs_now * 8, (size_t)L.R, cudaMemcpyDeviceToHost,
+                                      copy_st);
+            if (e == cudaSuccess) e = cudaEventRecord(sent[buf], copy_st);
+            if (e != cudaSuccess) { h->last_cuda = (int)e; rc = FCSIM_ECUDA; }
+            rec0 += recs_now;
+        }
+        if (rc == FCSIM_OK && cudaStreamSynchronize(run_st) != cudaSuccess) rc = FCSIM_ECUDA;
+    }
+    if (rc == FCSIM_OK) rc = fcsim_stats(h, run_st, host_counters, per_group_out);
     if (rc == FCSIM_OK) {
         cudaError_t e = cudaSuccess;
-        if (host_trace && sz.trace) e = cudaMemcpy(host_trace, b.trace, sz.trace, cudaMemcpyDeviceToHost);
+        if (win_recs > 0) {
+            e = cudaStreamSynchronize(copy_st);
+            // records of slots that were not run read as zero, as in a freshly created trace buffer
+            if (e == cudaSuccess && recs_run < L.n_rec)
+                for (long long r = 0; r < L.R; ++r)
+                    std::memset(static_cast<unsigned char*>(host_trace) + ((size_t)r * L.n_rec + (size_t)recs_run) * 8, 0,
+                                (size_t)(L.n_rec - recs_run) * 8);
+        } else if (host_trace && sz.trace) {
+            e = cudaMemcpy(host_trace, b.trace, sz.trace, cudaMemcpyDeviceToHost);
+        }
         if (e == cudaSuccess && host_hist && sz.hist) e = cudaMemcpy(host_hist, b.hist, sz.hist, cudaMemcpyDeviceToHost);
         if (e == cudaSuccess && host_complog && sz.complog)
             e = cudaMemcpy(host_complog, b.complog, sz.complog, cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) rc = FCSIM_ECUDA;
     }
-    if (h) fcsim_destroy(h);
     free_all();
     return rc;
 }

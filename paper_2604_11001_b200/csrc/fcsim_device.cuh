@@ -88,7 +88,9 @@ struct Params {
     uint32_t key0, key1;
     int32_t n_classes, n_groups, n_replicas;  // n_groups: entries of `groups`
     int32_t n_work;               // replicas this launch advances (those of the groups in `groups`)
-    int32_t trace_stride, n_rec, hist_bins, hist_shift, complog_cap;
+    int32_t trace_stride, n_rec, hist_bins, hist_shift, complog_cap;  // n_rec: records a trace row holds
+    int32_t rec_base;             // index of the first record the trace rows hold (0 unless the buffer is a window
+                                  // on the horizon that the host moves from launch to launch)
     int32_t t0, n_steps;
     const uint32_t* pool;         // all thresholds
     const uint4* gpool;           // guide records {k0, thresholds k0, k0+1, k0+2}, one per bucket of u
@@ -257,7 +259,7 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define RING(i) checked_ref(ring, (i), Acap, __LINE__, p.debug, r)
 #define STATE(i) checked_ref(state, (i), Acap, __LINE__, p.debug, r)
 #define STAGE(i) checked_ref(stage, (i), S, __LINE__, p.debug, r)
-#define TROW(i) checked_ref(trow, (i), p.n_rec, __LINE__, p.debug, r)
+#define TROW(i) checked_ref(trow + p.rec_base, (long long)(i) - p.rec_base, p.n_rec, __LINE__, p.debug, r)
 #define LROW(i) checked_ref(lrow, (i), p.complog_cap, __LINE__, p.debug, r)
 #define HROW(i) checked_ref(hrow, (i), p.hist_bins, __LINE__, p.debug, r)
 #else
@@ -282,7 +284,10 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 // (the host picks it when the longest output length is short next to the active set's storage).
 // kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80).  The host
 // asks the occupancy calculator about both.
-template <int kPol, int kMinCtas, int kRec>
+// kBulk: the whole-prompt first-come-first-served policies (0, 1, 3) first try to activate several queue heads at
+// once; the host asks for it when two or more requests arrive (and may be activated) per slot on average.  With
+// fewer the extra code only costs.
+template <int kPol, int kMinCtas, int kRec, bool kBulk>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     constexpr bool kExt = kPol >= 4;
     constexpr bool kMcProfile = kPol == 6;  // MC benchmark, projection per future slot
@@ -453,8 +458,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         // with one 256-byte bulk copy issued by lane 0, when the row's address allows it
         int2* tstage = reinterpret_cast<int2*>(my + p.tstage_off);
         const bool staged = p.tstage_off != 0 && tracing &&
-                            ((reinterpret_cast<uintptr_t>(p.trace + (size_t)r * p.n_rec) & 15u) == 0);
-        int2* trow = (kRec != 0 && p.trace) ? p.trace + (size_t)r * p.n_rec : nullptr;
+                            (((reinterpret_cast<uintptr_t>(p.trace + (size_t)r * p.n_rec) - (size_t)p.rec_base * 8u) & 15u) == 0);
+        // trow[rec] is record rec of this replica: rec_base <= rec < rec_base + n_rec
+        int2* trow = (kRec != 0 && p.trace) ? p.trace + ((long long)r * p.n_rec - p.rec_base) : nullptr;
         int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
         int2* lrow = (kRec == 2 && p.complog) ? p.complog + (size_t)r * p.complog_cap : nullptr;
 
@@ -672,6 +678,69 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         // towards the tail and the pick takes the freed place next to the active range.
                         bool gate_hit = false, budget_hit = false, storage_hit = false;
                         const int32_t* bk = p.bclass + grp.bclass_off;
+                        if (nQ > 0 && nQ <= 32 && p.n_classes <= 8) {
+                            // Short queue: all picks of the slot at once (lane = waiting request).  A request is
+                            // picked when fewer than b_k requests of its class wait ahead of it; the picks are
+                            // activated class by class, in queue order within a class.  Taken only when every pick
+                            // passes the gate, the token budget and the storage bound (the usage is largest with all
+                            // of them in, so one test covers every prefix); otherwise the loop below decides pick by pick.
+                            const bool in = lane < nQ;
+                            const uint64_t e = qwin[(qh + (uint32_t)lane) & 63u];
+                            const int cls = in ? entry_cls(e) : -1;
+                            int rank = 0, before = 0, npick = 0, mytake = 0;
+                            bool picked = false;
+                            for (int kc = 0; kc < p.n_classes; ++kc) {
+                                const uint32_t mk = __ballot_sync(FULL, cls == kc);
+                                const int take = min(__popc(mk), __ldg(bk + kc));
+                                if (cls == kc) {
+                                    rank = __popc(mk & lt_mask);
+                                    picked = rank < take;
+                                    before = npick;
+                                }
+                                if (lane == kc) mytake = take;
+                                npick += take;
+                            }
+                            const int l = entry_l(e);
+                            const int tot_l = __reduce_add_sync(FULL, picked ? l : 0);
+                            if (npick > 0 && nP + npick <= Acap && G + tot_l + npick <= M &&
+                                (kinf || npick == 1 || tot_l <= R)) {
+                                const int dest = nP + before + rank;  // place in the active range
+                                const uint32_t sw = picked ? (uint32_t)(t + entry_o(e) - 1) : kNoFin;
+                                const uint32_t pm = __ballot_sync(FULL, picked);
+                                // the requests left behind keep their order and close ranks towards the tail
+                                const uint32_t stay_seq = qh + (uint32_t)(npick + lane - __popc(pm & lt_mask));
+                                __syncwarp();  // every lane holds its entry: the window may be overwritten
+                                if (picked) {
+                                    RING(WA(shead + dest)) = e;
+                                    STATE(WA(shead + dest)) = sw;
+                                } else if (in) {
+                                    q_put(stay_seq, e);
+                                }
+                                if (lane < p.n_classes) qcnt[lane] -= (uint32_t)mytake;
+                                const int c0 = nP >> bsh;
+                                const bool lo_part = (dest >> bsh) == c0;
+                                const uint32_t m0 = __reduce_min_sync(FULL, lo_part ? sw : kNoFin);
+                                const uint32_t m1 = __reduce_min_sync(FULL, lo_part ? kNoFin : sw);
+                                if (lane == c0) cmin = min(cmin, m0);
+                                if (lane == c0 + 1) cmin = min(cmin, m1);
+                                next_fin = min(next_fin, min(m0, m1));
+                                G += tot_l + npick;
+                                if (!kinf) R = max(0, R - tot_l);
+                                Ndec += npick;
+                                nP += npick;
+                                a = npick;
+                                CADD(C_PREFILL_TOKENS, tot_l);
+                                qh += (uint32_t)npick;
+                                nQ -= npick;
+                                __syncwarp();
+                                if (qh - wseq >= 32u) {  // the window moves on as in q_pop
+                                    wseq += 32u;
+                                    q_fill(wseq + 32u);
+                                }
+                                q_e = 0;
+                                break;
+                            }
+                        }
                         for (int kc = 0; kc < p.n_classes && !storage_hit; ++kc) {
                             const int b_k = __ldg(bk + kc);
                             for (int ak = 0; ak < b_k && qcnt[kc] > 0; ++ak) {
@@ -726,6 +795,55 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         q_e = 0;
                         break;
                     } else {
+                    if constexpr (kBulk && (policy <= 1 || policy == 3)) {
+                        // Several queue heads at once (lane = candidate): the heads that the sequential rule would
+                        // admit one after the other are the leading run of candidates whose cumulative need still
+                        // passes the gate and whose cumulative prompt tokens still fit the slot's token room (the
+                        // slot's first admission is exempt).  The candidate that ends the run is left to the
+                        // sequential loop below, which counts the reason.
+                        int want = min(min(cap - a, nQ), Acap - nP);
+                        if (want >= 2) {
+                            want = min(want, 32);
+                            const bool in = lane < want;
+                            const uint64_t e = qwin[(qh + (uint32_t)lane) & 63u];  // the first 32 queue places are in the window
+                            const int l = entry_l(e);
+                            const int pre = warp_incl_scan(in ? l + 1 : 0, lane);  // tokens the slot's usage grows by
+                            const int pre_l = pre - (lane + 1);                    // prompt tokens of candidates 0 .. lane
+                            const bool ok = in && G + pre <= admit_limit && (kinf || (a == 0 && lane == 0) || pre_l <= R);
+                            const uint32_t okm = __ballot_sync(FULL, ok);
+                            const int n = (okm == FULL) ? 32 : __ffs((int)~okm) - 1;
+                            if (n > 0) {
+                                const uint32_t sw = (lane < n) ? (uint32_t)(t + entry_o(e) - 1) : kNoFin;
+                                if (lane < n) {
+                                    RING(WA(shead + nP + lane)) = e;
+                                    STATE(WA(shead + nP + lane)) = sw;
+                                }
+                                // the new entries lie in at most two watched stretches of the active range
+                                const int c0 = nP >> bsh;
+                                const bool lo_part = ((nP + lane) >> bsh) == c0;
+                                const uint32_t m0 = __reduce_min_sync(FULL, lo_part ? sw : kNoFin);
+                                const uint32_t m1 = __reduce_min_sync(FULL, lo_part ? kNoFin : sw);
+                                if (lane == c0) cmin = min(cmin, m0);
+                                if (lane == c0 + 1) cmin = min(cmin, m1);
+                                next_fin = min(next_fin, min(m0, m1));
+                                const int tot = __shfl_sync(FULL, pre, n - 1);
+                                G += tot;
+                                if (!kinf) R = max(0, R - (tot - n));
+                                Ndec += n;
+                                nP += n;
+                                a += n;
+                                CADD(C_PREFILL_TOKENS, tot - n);
+                                qh += (uint32_t)n;
+                                nQ -= n;
+                                q_e = 0;
+                                __syncwarp();
+                                if (qh - wseq >= 32u) {  // the window moves on as in q_pop
+                                    wseq += 32u;
+                                    q_fill(wseq + 32u);
+                                }
+                            }
+                        }
+                    }
                     while (a < cap && nQ > 0) {
                         if (nP == Acap) {
                             if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room

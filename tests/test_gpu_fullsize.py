@@ -176,3 +176,27 @@ def test_horizon_at_the_24_bit_limit():
     # 32 768 slots whose 32-bit partial sums are folded into the int64 counters
     cfg = wl.config1(replicas=2, T=(1 << 24) - 1).with_(trace_stride=4096, complog_cap=4096, hist_shift=3)
     _run_full(cfg, (1 << 24) - 1, [0, 1])
+
+
+def test_host_buffer_entry_point_streams_a_large_trace():
+    # 8192 replicas x 8000 slots: a 524 MB trace leaves the device in windows of 2048 records per replica while the
+    # run goes on (four windows, the last one partial); every output word against the CPU checker.  The second
+    # call stops 1000 slots before the horizon: the records of the slots not run must read as zero.
+    from paper_2604_11001_b200 import binding as fb
+    cfg = wl.config2(replicas=4096, T=8000)
+    assert fb.fcsim_query_sizes(cfg)["trace"] >= 256 << 20
+    ref = orc.run(cfg, threads=16)
+    host = fb.host_output_arrays(cfg, pinned=True)
+    out = fb.fcsim_simulate_host(cfg, out=host)
+    assert (out["counters"] == ref["counters"]).all()
+    assert (out["trace"] == ref["trace"]).all()
+    assert (out["hist"] == ref["hist"]).all()
+    n = ref["counters"][:, I["n_logged"]]
+    live = np.arange(cfg.complog_cap)[None, :] < n[:, None]
+    assert ((out["complog"] == ref["complog"]).all(axis=2) | ~live).all()
+    host["trace"][:] = -1
+    part = fb.fcsim_simulate_host(cfg, 7000, out=host)
+    assert (part["trace"][:, :7000] == ref["trace"][:, :7000]).all()
+    assert (part["trace"][:, 7000:] == 0).all()
+    short = orc.run(cfg, 0, 64, 7000, threads=16)
+    assert (part["counters"][:64] == short["counters"]).all()
