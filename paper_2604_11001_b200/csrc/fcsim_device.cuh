@@ -517,6 +517,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             next_fin = __reduce_min_sync(FULL, cmin);
         };
         rebuild_minima();
+        auto squeeze_now = [&]() {
+            compact();
+            rebuild_minima();
+        };
         if ((kExt && policy == 4)) {  // Algorithm 1 picks per class: count the waiting requests of every class
             for (int c = lane; c < p.n_classes; c += 32) qcnt[c] = 0;
             __syncwarp();
@@ -654,30 +658,23 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     __syncwarp();
                 }
 
-                // ---- completed entries are squeezed out when too many have piled up, before the active range
-                //      runs out of storage, and before the whole active range is sent back (alpha-protection)
-                bool squeeze = nD > 0 && (nD >= kCompactAt || (policy == 3 && G > M) ||
-                                          ((kExt && policy == 4) && nP + nQ > Acap));
-
                 // ---- activation (Alg. 2 inner loop): FIFO, at most B_t under flow control
                 int a = 0;
                 const int cap = (policy == 0) ? B_t : 0x7fffffff;
-                if (gate_closed && !squeeze) {
+                if (gate_closed) {
                     if (cap > 0) CADD(C_GATE_BLOCKED, 1);
-                } else
-                for (;;) {
-                    if (squeeze) {
-                        __syncwarp();  // state words written by lane 0 during this slot's activations
-                        compact();
-                        rebuild_minima();
-                        squeeze = false;
-                    }
+                } else {
+                    do {
                     if constexpr (policy == 4) {
                         // Algorithm 1: for every class k, up to b_k waiting requests of that class, oldest first.
                         // The pick leaves the middle of the queue: the entries ahead of it move one place
                         // towards the tail and the pick takes the freed place next to the active range.
                         bool gate_hit = false, budget_hit = false, storage_hit = false;
                         const int32_t* bk = p.bclass + grp.bclass_off;
+                        if (nD > 0 && nP + nQ > Acap) {  // the picks below take the storage bound at face value
+                            __syncwarp();
+                            squeeze_now();
+                        }
                         if (nQ > 0 && nQ <= 32 && p.n_classes <= 8) {
                             // Short queue: all picks of the slot at once (lane = waiting request).  A request is
                             // picked when fewer than b_k requests of its class wait ahead of it; the picks are
@@ -846,7 +843,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     }
                     while (a < cap && nQ > 0) {
                         if (nP == Acap) {
-                            if (nD > 0) { squeeze = true; break; }  // storage, not the model's bound: make room
+                            if (nD > 0) {  // storage, not the model's bound: make room
+                                __syncwarp();  // state words written by lane 0 during this slot's activations
+                                squeeze_now();
+                                continue;
+                            }
                             CADD(C_ACAP_BLOCKED, 1); status |= 1u; break;
                         }
                         if (q_e == 0) q_e = qwin[qh & 63u];  // the head is always inside the window
@@ -977,10 +978,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         a++;
                         CADD(C_PREFILL_TOKENS, g);
                     }
-                    if (!squeeze) break;
                     }
+                    } while (false);
+                    if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
                 }
-                if (a > 0) { CADD(C_ADMITTED, a); __syncwarp(); }
 
                 // ---- overflow: evict the most recently activated until the slot fits (LIFO, Section 3.3);
                 //      evicted requests lose all progress (or, in the variant that keeps the generated tokens,
@@ -991,8 +992,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     int nev = 0, wasted = 0;
                     if (policy == 3) {
                         // alpha-protection greedy (Section 4.1): every active request goes back to the queue.
-                        // Completed entries were squeezed out above, so the whole active range is live and is
+                        // Completed entries are squeezed out first, so the whole active range is live and is
                         // copied, in order, in front of the queue head.
+                        if (nD > 0) {
+                            __syncwarp();
+                            compact();
+                        }
                         long long kept_w = 0;
                         const uint32_t nqh = qh - (uint32_t)nP;
                         wseq = nqh;  // the window restarts at the new head (reloaded below)
@@ -1203,6 +1208,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             n_logged = min(p.complog_cap, n_logged + ndone);
                         }
                         __syncwarp();
+                        // completed entries are squeezed out when enough have piled up (and whenever the storage
+                        // of the active range runs out, or the whole range is sent back)
+                        if (nD >= kCompactAt) squeeze_now();
                     }
                 }
 

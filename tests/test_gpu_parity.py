@@ -418,3 +418,33 @@ def test_standing_queue_of_200000_over_a_long_run():
     assert (c[:, I["q_final"]] == 200000).all() and (c[:, I["dropped"]] == 255 * 33000 - 200000).all()
     ref = orc.run(cfg, threads=2)
     assert_same(cfg, gpu, ref, 33000, "standing queue")
+
+
+def test_many_activations_per_slot():
+    # six arrivals per slot and a cache that serves about as many: the kernels that activate several queue heads
+    # at once are chosen; gate, token budget (with and without), storage bound and flow-control budget all end
+    # runs of activations, evictions push requests back in front of the window on the queue
+    for K, M, Acap in ((0, 1400, 200), (45, 3000, 200), (0, 1000, 200), (0, 100000, 48)):
+        cfg = wl.SimConfig(
+            M=M, K=K, T_max=700, Qcap=100, Acap=Acap, seed=91 + K, class_law=wl.table_from_pmf(0, [0.5, 0.5]),
+            prompt=(wl.uniform_table(1, 20), wl.uniform_table(5, 9)), decode=(wl.uniform_table(1, 30), wl.uniform_table(2, 12)),
+            arrivals=(wl.Arrivals((wl.poisson_table(6.0),)), wl.Arrivals((wl.poisson_table(3.0), wl.poisson_table(9.0)), (1 << 27, 1 << 28))),
+            groups=(wl.Group(wl.POLICY_FLOW, b_fp=wl.b_to_fp(5.5), n_replicas=5),
+                    wl.Group(wl.POLICY_GREEDY, n_replicas=5, arrivals_id=1),
+                    wl.Group(wl.POLICY_ALPHA, n_replicas=5, m_admit=int(0.8 * M)),
+                    wl.Group(wl.POLICY_GREEDY, n_replicas=4, preempt_keep=1, rng_replica_base=40),
+                    wl.Group(wl.POLICY_CLASSFLOW, n_replicas=5, b_class=(3, 4)),
+                    wl.Group(wl.POLICY_FLOW, b_fp=wl.b_to_fp(40.0), n_replicas=3, arrivals_id=1)),
+            trace_stride=1, hist_bins=64, hist_shift=1, complog_cap=6000)
+        ref = orc.run(cfg, threads=4)
+        c = ref["counters"]
+        assert c[:, orc.CIDX["admitted"]].min() > 2 * 700
+        if M == 1000:
+            assert c[:, orc.CIDX["evictions"]].sum() > 100 and c[:, orc.CIDX["gate_blocked_steps"]].min() > 50
+        if K:
+            assert c[:, orc.CIDX["budget_blocked_steps"]].sum() > 100
+        if Acap == 48:
+            assert c[:, orc.CIDX["acap_blocked_steps"]].sum() > 0
+        gpu = run_gpu(cfg, pieces=[333, 367])
+        assert_same(cfg, gpu, ref, 700, f"many activations K={K} M={M} Acap={Acap}")
+        assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 700, ref["complog"])
