@@ -427,6 +427,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         unsigned long long sumU = 0;
         uint32_t sumN = 0, tokgen = 0, arrived = 0, accepted = 0;
         int maxU = 0, maxQ = 0;
+        int nTot = nP - nD + nQ;  // requests in the system: changes only when requests arrive or complete
         int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
         uint64_t q_e = 0;  // the queue head's entry when known, else 0 (saves shared-memory reads in blocked slots)
         // Whole-prompt policies: once the headroom gate has refused the queue head, it keeps refusing it until
@@ -608,6 +609,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
                     }
                     nQ += acc;
+                    nTot += acc;
                     accepted += acc;
                     __syncwarp();
                 }
@@ -987,6 +989,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 //      evicted requests lose all progress (or, in the variant that keeps the generated tokens,
                 //      only their place in the cache) and are again the head of the queue
                 if (G > M) {
+                    maxU = max(maxU, U);  // the last slot's usage, before this slot's evictions lower it
                     gate_closed = false;
                     CADD(C_OVERFLOW_STEPS, 1);
                     int nev = 0, wasted = 0;
@@ -1099,8 +1102,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 tokgen += Ndec;
                 U = G;
                 sumU += (unsigned)G;
-                maxU = max(maxU, G);
-                sumN += nP - nD + nQ;
+                sumN += nTot;
 
                 // ---- retire the requests that generated their last token in this slot: their statistics
                 //      are taken now, their entries are only marked and squeezed out later in bulk
@@ -1198,8 +1200,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     if (kPol == 5 && npend > 0) mc_release();
                     next_fin = __reduce_min_sync(FULL, cmin);
                     if (ndone > 0) {
+                        // the usage only falls when requests leave or are evicted: its maximum is taken there
+                        maxU = max(maxU, G);
                         gate_closed = false;
                         nD += ndone;
+                        nTot -= ndone;
                         Ndec -= ndone;
                         completed += ndone;
                         U -= __reduce_add_sync(FULL, sum_lo);
@@ -1292,7 +1297,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         CADD(C_SUM_W_COMPLETED, warp_sum64((long long)acc_w));
         CADD(C_COMPLETED_TOKENS, warp_sum64((long long)acc_o));
         CMAX(C_MAX_LAT, __reduce_max_sync(FULL, acc_maxlat));
-        CMAX(C_MAX_U, maxU);
+        CMAX(C_MAX_U, max(maxU, U));  // U: the usage of the last slot if nothing left in it
         CMAX(C_MAX_Q, maxQ);
         CSET(C_STEPS_DONE, t_end);
         CSET(C_STATUS, status);
