@@ -266,9 +266,13 @@ int fcsim_debug_read(fcsim_t* h, uint32_t out[8]);
 int fcsim_is_checked_build(void);
 const char* fcsim_strerror(int code);
 
-/* Whole job with HOST buffers: allocates device buffers (cudaMalloc), runs slots 1..n_steps, copies the
- * outputs to the given HOST arrays (each may be NULL; shapes as in fcsim_buffers with T_max = cfg->T_max)
- * and frees the device memory.  Synchronous. */
+/* Whole job with HOST buffers: allocates device memory (one cudaMalloc), runs slots 1..n_steps, copies the
+ * outputs to the given HOST arrays (each may be NULL; shapes as in fcsim_buffers with T_max = cfg->T_max; trace
+ * records of slots that were not run read as zero) and frees the device memory.  Synchronous.
+ * A trace of 256 MB or more does not wait for the end of the run: the device holds only two windows of the
+ * horizon (2048 records per replica or more each), and every filled window is copied into the caller's rows
+ * with one strided copy on a second stream while the kernels fill the other.  The copies overlap the run only
+ * when host_trace is page-locked memory; with pageable memory the result is the same, later. */
 int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcsim_counters* host_counters,
                         void* host_trace, void* host_hist, void* host_complog, fcsim_summary* per_group_out);
 

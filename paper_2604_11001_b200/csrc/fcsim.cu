@@ -509,6 +509,7 @@ struct fcsim {
     Layout L;
     fcsim_buffers buf;
     Params params;
+    void* d_blob = nullptr;              // one allocation holding everything below up to d_work
     uint32_t* d_pool = nullptr;
     uint4* d_gpool = nullptr;
     int32_t* d_bclass = nullptr;
@@ -682,24 +683,31 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         pl.pg_cnt = (int)pgrps.size() - pl.pg_off;
         if (pl.pg_cnt > 0) h->launches.push_back(pl);
     }
-    CUDA_TRY(h, cudaMalloc(&h->d_bclass, bclass.size() * sizeof(int32_t)));
-    CUDA_TRY(h, cudaMemcpy(h->d_bclass, bclass.data(), bclass.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
     if (gpool.empty()) gpool.push_back(make_uint4(0, 0, 0, 0));
     if (gpool.size() > (size_t)0x3fffff) return FCSIM_ECAP;  // a guide's first record is a 22-bit index
-    CUDA_TRY(h, cudaMalloc(&h->d_gpool, gpool.size() * sizeof(uint4)));
-    CUDA_TRY(h, cudaMemcpy(h->d_gpool, gpool.data(), gpool.size() * sizeof(uint4), cudaMemcpyHostToDevice));
-    CUDA_TRY(h, cudaMalloc(&h->d_pool, pool.size() * sizeof(uint32_t)));
-    CUDA_TRY(h, cudaMalloc(&h->d_tables, tables.size() * sizeof(DevTable)));
-    CUDA_TRY(h, cudaMalloc(&h->d_arrivals, arrs.size() * sizeof(DevArrivals)));
-    CUDA_TRY(h, cudaMalloc(&h->d_groups, grps.size() * sizeof(DevGroup)));
-    CUDA_TRY(h, cudaMalloc(&h->d_pgroups, pgrps.size() * sizeof(DevGroup)));
-    CUDA_TRY(h, cudaMemcpy(h->d_pgroups, pgrps.data(), pgrps.size() * sizeof(DevGroup), cudaMemcpyHostToDevice));
-    CUDA_TRY(h, cudaMalloc(&h->d_work, 16 * sizeof(unsigned int)));
-    CUDA_TRY(h, cudaMemset(h->d_work, 0, 16 * sizeof(unsigned int)));
-    CUDA_TRY(h, cudaMemcpy(h->d_pool, pool.data(), pool.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
-    CUDA_TRY(h, cudaMemcpy(h->d_tables, tables.data(), tables.size() * sizeof(DevTable), cudaMemcpyHostToDevice));
-    CUDA_TRY(h, cudaMemcpy(h->d_arrivals, arrs.data(), arrs.size() * sizeof(DevArrivals), cudaMemcpyHostToDevice));
-    CUDA_TRY(h, cudaMemcpy(h->d_groups, grps.data(), grps.size() * sizeof(DevGroup), cudaMemcpyHostToDevice));
+    // one device allocation and one copy for all the tables (a handle is often created for a short run)
+    struct Part { const void* src; size_t bytes; void** dst; };
+    const Part parts[] = {
+        {gpool.data(), gpool.size() * sizeof(uint4), reinterpret_cast<void**>(&h->d_gpool)},
+        {pool.data(), pool.size() * sizeof(uint32_t), reinterpret_cast<void**>(&h->d_pool)},
+        {tables.data(), tables.size() * sizeof(DevTable), reinterpret_cast<void**>(&h->d_tables)},
+        {arrs.data(), arrs.size() * sizeof(DevArrivals), reinterpret_cast<void**>(&h->d_arrivals)},
+        {grps.data(), grps.size() * sizeof(DevGroup), reinterpret_cast<void**>(&h->d_groups)},
+        {pgrps.data(), pgrps.size() * sizeof(DevGroup), reinterpret_cast<void**>(&h->d_pgroups)},
+        {bclass.data(), bclass.size() * sizeof(int32_t), reinterpret_cast<void**>(&h->d_bclass)},
+        {nullptr, 16 * sizeof(unsigned int), reinterpret_cast<void**>(&h->d_work)},  // work counters + debug record: zero
+    };
+    size_t total = 0;
+    for (const Part& q : parts) total += align_up(q.bytes, 256);
+    std::vector<unsigned char> blob(total, 0);
+    CUDA_TRY(h, cudaMalloc(&h->d_blob, total));
+    size_t off = 0;
+    for (const Part& q : parts) {
+        if (q.src) std::memcpy(blob.data() + off, q.src, q.bytes);
+        *q.dst = static_cast<unsigned char*>(h->d_blob) + off;
+        off += align_up(q.bytes, 256);
+    }
+    CUDA_TRY(h, cudaMemcpy(h->d_blob, blob.data(), total, cudaMemcpyHostToDevice));
     h->table_bytes = pool.size() * 4 + tables.size() * sizeof(DevTable) + arrs.size() * sizeof(DevArrivals) +
                      grps.size() * sizeof(DevGroup);
     return FCSIM_OK;
@@ -707,19 +715,12 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
 
 static void release(fcsim* h) {
     if (!h) return;
-    cudaFree(h->d_pool);
-    cudaFree(h->d_gpool);
-    cudaFree(h->d_bclass);
-    cudaFree(h->d_tables);
-    cudaFree(h->d_arrivals);
-    cudaFree(h->d_groups);
-    cudaFree(h->d_pgroups);
+    cudaFree(h->d_blob);  // all the tables
     for (PolicyLaunch& pl : h->launches) {
         if (pl.done) cudaEventDestroy(pl.done);
         if (pl.side) cudaStreamDestroy(pl.side);
     }
     if (h->fork) cudaEventDestroy(h->fork);
-    cudaFree(h->d_work);
     delete h;
 }
 
@@ -765,8 +766,13 @@ static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_
     };
     cudaError_t e = cudaGetDevice(&h->device);
     if (e != cudaSuccess) return fail(FCSIM_ECUDA);
-    cudaDeviceProp prop;
-    e = cudaGetDeviceProperties(&prop, h->device);
+    // three attribute queries (the whole property structure takes far longer to fill)
+    struct { int multiProcessorCount, sharedMemPerMultiprocessor, sharedMemPerBlockOptin; } prop = {0, 0, 0};
+    e = cudaDeviceGetAttribute(&prop.multiProcessorCount, cudaDevAttrMultiProcessorCount, h->device);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&prop.sharedMemPerMultiprocessor, cudaDevAttrMaxSharedMemoryPerMultiprocessor, h->device);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&prop.sharedMemPerBlockOptin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
     if (e != cudaSuccess) return fail(FCSIM_ECUDA);
     h->sm_count = prop.multiProcessorCount;
     try {
@@ -1188,9 +1194,10 @@ extern "C" int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcs
     cudaStream_t run_st = nullptr, copy_st = nullptr;
     cudaEvent_t filled[2] = {nullptr, nullptr}, sent[2] = {nullptr, nullptr};
     fcsim_t* h = nullptr;
+    void* arena = nullptr;  // one device allocation for all the buffers
     auto free_all = [&]() {
         if (h) fcsim_destroy(h);
-        for (void** s : slots) cudaFree(*s);
+        cudaFree(arena);
         for (int i = 0; i < 2; ++i) {
             if (filled[i]) cudaEventDestroy(filled[i]);
             if (sent[i]) cudaEventDestroy(sent[i]);
@@ -1198,10 +1205,14 @@ extern "C" int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcs
         if (run_st) cudaStreamDestroy(run_st);
         if (copy_st) cudaStreamDestroy(copy_st);
     };
-    for (int i = 0; i < 6; ++i) {
-        if (bytes[i] && cudaMalloc(slots[i], bytes[i]) != cudaSuccess) {
-            free_all();
-            return FCSIM_ECUDA;
+    size_t total = 0;
+    for (int i = 0; i < 6; ++i) total += align_up(bytes[i], 256);
+    if (cudaMalloc(&arena, std::max<size_t>(total, 256)) != cudaSuccess) return FCSIM_ECUDA;
+    {
+        size_t off = 0;
+        for (int i = 0; i < 6; ++i) {
+            if (bytes[i]) *slots[i] = static_cast<unsigned char*>(arena) + off;
+            off += align_up(bytes[i], 256);
         }
     }
     rc = create_handle(cfg, &b, &h, (int)win_recs);
