@@ -268,7 +268,9 @@ const char* fcsim_strerror(int code);
 
 /* Whole job with HOST buffers: allocates device memory (one cudaMalloc), runs slots 1..n_steps, copies the
  * outputs to the given HOST arrays (each may be NULL; shapes as in fcsim_buffers with T_max = cfg->T_max; trace
- * records of slots that were not run read as zero) and frees the device memory.  Synchronous.
+ * records of slots that were not run read as zero; of a completion-log row only the first n_logged entries are
+ * meaningful, and entries beyond the longest row's n_logged may be left untouched) and frees the device memory.
+ * Synchronous.
  * A trace of 256 MB or more does not wait for the end of the run: the device holds only two windows of the
  * horizon (2048 records per replica or more each), and every filled window is copied into the caller's rows
  * with one strided copy on a second stream while the kernels fill the other.  The copies overlap the run only

@@ -345,11 +345,18 @@ __global__ void __launch_bounds__(256) latency_digit_kernel(const int2* __restri
         }
         __syncthreads();
     };
+    // Latencies cluster: when all the lanes of a warp that count hit one bin (the rule for the high digit, and for
+    // constant lengths) one lane adds their number; otherwise every lane adds one (bins spread, few collisions).
     auto count = [&](unsigned int* table, bool mine, unsigned int bin) {
         const unsigned int voters = __ballot_sync(0xffffffffu, mine);
-        if (mine) {
-            const unsigned int peers = __match_any_sync(voters, bin);
-            if ((threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(table + bin, (unsigned)__popc(peers));
+        if (voters == 0u) return;
+        const int leader = __ffs(voters) - 1;
+        const unsigned int lead_bin = __shfl_sync(0xffffffffu, bin, leader);
+        const bool same = __all_sync(0xffffffffu, !mine || bin == lead_bin);
+        if (same) {
+            if ((int)(threadIdx.x & 31) == leader) atomicAdd(table + bin, (unsigned)__popc(voters));
+        } else if (mine) {
+            atomicAdd(table + bin, 1u);
         }
     };
     for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
@@ -383,7 +390,8 @@ __global__ void __launch_bounds__(256) latency_digit_kernel(const int2* __restri
                         count(sh, have, v >> kSelBits);
                     } else {
                         count(sh, have && (v >> kSelBits) == hi95, v & (kSelBins - 1));
-                        count(sh + kSelBins, have && (v >> kSelBits) == hi99, v & (kSelBins - 1));
+                        // both ranks in one high digit (the rule): the first table serves both
+                        if (hi99 != hi95) count(sh + kSelBins, have && (v >> kSelBits) == hi99, v & (kSelBins - 1));
                     }
                 }
             }
@@ -406,7 +414,9 @@ __global__ void __launch_bounds__(256) latency_select_kernel(const unsigned long
     constexpr int kPer = kSelBins / 256;
     long long* out = res + (size_t)g * kSelResultWords;
     for (int qi = 0; qi < 2; ++qi) {
-        const unsigned long long* row = tables + ((size_t)g * (kPass == 1 ? 1 : 2) + (kPass == 1 ? 0 : qi)) * kSelBins;
+        // pass 2 fills the second table only when the two ranks differ in the high digit
+        const int tab = (kPass == 1 || out[3] == out[5]) ? 0 : qi;
+        const unsigned long long* row = tables + ((size_t)g * (kPass == 1 ? 1 : 2) + tab) * kSelBins;
         unsigned long long mine = 0;
         for (int k = 0; k < kPer; ++k) mine += row[tid * kPer + k];
         part[tid] = mine;
@@ -457,10 +467,10 @@ static std::mutex g_kernel_attr_mutex;
 // activation of several queue heads at once.
 template <int kPol, int kCtas>
 static step_kernel_t step_kernel_for(int rec, bool bulk) {
-    constexpr bool kFifo = kPol <= 1 || kPol == 3;
+    constexpr bool kFifo = kPol <= 1 || kPol == 3 || kPol == 6;
     constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 .. 6 uninstantiated
     if (kFifo && bulk) {
-        if (rec == 2) return fcsim_step_kernel<kP, kCtas, 2, kFifo>;
+        if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, kFifo>;
         if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, kFifo>;
         return fcsim_step_kernel<kP, kCtas, 0, kFifo>;
     }
@@ -1272,8 +1282,17 @@ extern "C" int fcsim_simulate_host(const fcsim_config* cfg, int32_t n_steps, fcs
             e = cudaMemcpy(host_trace, b.trace, sz.trace, cudaMemcpyDeviceToHost);
         }
         if (e == cudaSuccess && host_hist && sz.hist) e = cudaMemcpy(host_hist, b.hist, sz.hist, cudaMemcpyDeviceToHost);
-        if (e == cudaSuccess && host_complog && sz.complog)
-            e = cudaMemcpy(host_complog, b.complog, sz.complog, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && host_complog && sz.complog) {
+            // rows are rarely full: with the counters on the host only the longest logged prefix of the rows travels
+            long long longest = cfg->complog_cap;
+            if (host_counters) {
+                longest = 0;
+                for (long long r = 0; r < L.R; ++r) longest = std::max<long long>(longest, host_counters[r].n_logged);
+            }
+            if (longest > 0)
+                e = cudaMemcpy2D(host_complog, (size_t)cfg->complog_cap * 8, b.complog, (size_t)cfg->complog_cap * 8,
+                                 (size_t)longest * 8, (size_t)L.R, cudaMemcpyDeviceToHost);
+        }
         if (e != cudaSuccess) rc = FCSIM_ECUDA;
     }
     free_all();

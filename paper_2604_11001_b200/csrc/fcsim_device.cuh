@@ -284,7 +284,7 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 // (the host picks it when the longest output length is short next to the active set's storage).
 // kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80).  The host
 // asks the occupancy calculator about both.
-// kBulk: the whole-prompt first-come-first-served policies (0, 1, 3) first try to activate several queue heads at
+// kBulk: the whole-prompt first-come-first-served policies (0, 1, 3, 6) first try to activate several queue heads at
 // once; the host asks for it when two or more requests arrive (and may be activated) per slot on average.  With
 // fewer the extra code only costs.
 template <int kPol, int kMinCtas, int kRec, bool kBulk>
@@ -794,7 +794,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         q_e = 0;
                         break;
                     } else {
-                    if constexpr (kBulk && (policy <= 1 || policy == 3)) {
+                    if constexpr (kBulk && (policy <= 1 || policy == 3 || policy == 6)) {
                         // Several queue heads at once (lane = candidate): the heads that the sequential rule would
                         // admit one after the other are the leading run of candidates whose cumulative need still
                         // passes the gate and whose cumulative prompt tokens still fit the slot's token room (the
@@ -810,7 +810,31 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             const int pre_l = pre - (lane + 1);                    // prompt tokens of candidates 0 .. lane
                             const bool ok = in && G + pre <= admit_limit && (kinf || (a == 0 && lane == 0) || pre_l <= R);
                             const uint32_t okm = __ballot_sync(FULL, ok);
-                            const int n = (okm == FULL) ? 32 : __ffs((int)~okm) - 1;
+                            int n = (okm == FULL) ? 32 : __ffs((int)~okm) - 1;
+                            if constexpr (kMcProfile) {
+                                // MC benchmark: the candidates of the run pass the future-memory test one after the
+                                // other (each is booked on the projection before the next is tested); the first
+                                // refusal ends the run
+                                int pass = 0;
+                                for (; pass < n; ++pass) {
+                                    const uint64_t ec = __shfl_sync(FULL, e, pass);
+                                    const int op_c = grp.mc_worst != 0 ? (tabs[1 + p.n_classes + entry_cls(ec)].vmin +
+                                                                          (int)tabs[1 + p.n_classes + entry_cls(ec)].n - 1)
+                                                                       : entry_o(ec);
+                                    const int a_c = entry_l(ec) - t + 1;
+                                    bool over = false;
+                                    for (int base = 0; base < op_c; base += 32) {
+                                        const int tau = t + base + lane;
+                                        over |= (base + lane < op_c) && (vproj[(uint32_t)tau & p.prof_mask] + a_c + tau > M);
+                                    }
+                                    if (__any_sync(FULL, over)) break;
+                                    for (int base = 0; base < op_c; base += 32) {
+                                        const int tau = t + base + lane;
+                                        if (base + lane < op_c) vproj[(uint32_t)tau & p.prof_mask] += a_c + tau;
+                                    }
+                                }
+                                n = pass;
+                            }
                             if (n > 0) {
                                 const uint32_t sw = (lane < n) ? (uint32_t)(t + entry_o(e) - 1) : kNoFin;
                                 if (lane < n) {
