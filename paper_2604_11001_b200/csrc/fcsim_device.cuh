@@ -458,7 +458,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         // staged variant: records go to shared memory (two buffers of 32) and every full block of 32 leaves
         // with one 256-byte bulk copy issued by lane 0, when the row's address allows it
         int2* tstage = reinterpret_cast<int2*>(my + p.tstage_off);
-        const bool staged = p.tstage_off != 0 && tracing &&
+        const bool staged = kRec == 2 && p.tstage_off != 0 && tracing &&  // the host asks for kRec 2 with it
                             (((reinterpret_cast<uintptr_t>(p.trace + (size_t)r * p.n_rec) - (size_t)p.rec_base * 8u) & 15u) == 0);
         // trow[rec] is record rec of this replica: rec_base <= rec < rec_base + n_rec
         int2* trow = (kRec != 0 && p.trace) ? p.trace + ((long long)r * p.n_rec - p.rec_base) : nullptr;
