@@ -466,35 +466,37 @@ static std::mutex g_kernel_attr_mutex;
 // exist in the run-time form only) and, for the whole-prompt first-come-first-served policies, with or without the
 // activation of several queue heads at once.
 template <int kPol, int kCtas>
-static step_kernel_t step_kernel_for(int rec, bool bulk) {
+static step_kernel_t step_kernel_for(int rec, bool bulk, bool lazy) {
     constexpr bool kFifo = kPol <= 1 || kPol == 3 || kPol == 6;
     constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 .. 6 uninstantiated
+    // lazily drawn arrivals: only the forms that record nothing per slot, without the several-heads step
+    if (kPol <= 3 && lazy && !bulk && rec == 0) return fcsim_step_kernel<kP, kCtas, 0, false, kPol <= 3>;
     if (kFifo && bulk) {
-        if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, kFifo>;
-        if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, kFifo>;
-        return fcsim_step_kernel<kP, kCtas, 0, kFifo>;
+        if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, kFifo, false>;
+        if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, kFifo, false>;
+        return fcsim_step_kernel<kP, kCtas, 0, kFifo, false>;
     }
-    if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, false>;
-    if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, false>;
-    return fcsim_step_kernel<kP, kCtas, 0, false>;
+    if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, false, false>;
+    if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, false, false>;
+    return fcsim_step_kernel<kP, kCtas, 0, false, false>;
 }
 template <int kPol>
-static step_kernel_t step_kernel_for(int ctas, int rec, bool bulk) {
+static step_kernel_t step_kernel_for(int ctas, int rec, bool bulk, bool lazy) {
     switch (ctas) {
-        case 5: return step_kernel_for<kPol, 5>(rec, bulk);
-        case 6: return step_kernel_for<kPol, 6>(rec, bulk);
-        default: return step_kernel_for<kPol, 7>(rec, bulk);
+        case 5: return step_kernel_for<kPol, 5>(rec, bulk, lazy);
+        case 6: return step_kernel_for<kPol, 6>(rec, bulk, lazy);
+        default: return step_kernel_for<kPol, 7>(rec, bulk, lazy);
     }
 }
-static step_kernel_t pick_step_kernel(int policy, int ctas, int rec, bool bulk) {
+static step_kernel_t pick_step_kernel(int policy, int ctas, int rec, bool bulk, bool lazy) {
     switch (policy) {
-        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(ctas, rec, bulk);
-        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(ctas, rec, bulk);
-        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(ctas, rec, bulk);
-        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec, bulk);
-        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec, bulk);
-        case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec, bulk);
-        case 6: return step_kernel_for<6>(ctas, rec, bulk);  // the MC benchmark with its projection per future slot
+        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec, bulk, lazy);
+        case 6: return step_kernel_for<6>(ctas, rec, bulk, lazy);  // the MC benchmark with its projection per future slot
         default: return nullptr;
     }
 }
@@ -507,6 +509,7 @@ struct PolicyLaunch {
     int pg_off = 0, pg_cnt = 0;   // its groups in d_pgroups
     int n_work = 0;               // replicas
     bool bulk = false;            // two or more requests arrive, and may be activated, per slot on average
+    bool lazy = false;            // at least twice as many requests arrive as the cache can serve: most are dropped
     int warps_per_block = 0, blocks_per_sm = 0, grid = 0;
     size_t smem_block = 0, tabcache_off = 0;
     cudaStream_t side = nullptr;  // null: the caller's stream
@@ -672,6 +675,7 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         pl.policy = pol;
         pl.pg_off = (int)pgrps.size();
         double most = 0.0;  // requests that arrive and may be activated per slot, the largest over the policy's groups
+        double busiest = 0.0;  // requests that arrive per slot, the largest over the policy's groups
         for (int g = 0; g < c->n_groups; ++g) {
             if (grps[g].policy != pol) continue;
             DevGroup d = grps[g];
@@ -685,11 +689,14 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
                 table_moments(A.count[st], &m, nullptr);
                 rate = std::max(rate, m);
             }
+            busiest = std::max(busiest, rate);
             if (pol == FCSIM_POLICY_FLOW) rate = std::min(rate, (double)d.b_fp / 65536.0);
             most = std::max(most, rate);
         }
         // activations per slot cannot outrun the arrivals, the flow-control rate or what the cache can serve
         pl.bulk = std::min(most, cap_rate) >= 2.0;
+        // heavy overload with a waiting room long enough to hide the head: arrivals are drawn when they get there
+        pl.lazy = busiest >= 2.0 * cap_rate && c->Qcap >= 128;
         pl.pg_cnt = (int)pgrps.size() - pl.pg_off;
         if (pl.pg_cnt > 0) h->launches.push_back(pl);
     }
@@ -818,7 +825,7 @@ static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_
             }
             for (int ctas = 5; ctas <= 7; ++ctas) {
                 step_kernel_t k = pick_step_kernel(pl.policy == FCSIM_POLICY_MC && L.prof_mask ? 6 : pl.policy, ctas, rec,
-                                                   pl.bulk);
+                                                   pl.bulk, pl.lazy);
                 if (!k) return fail(FCSIM_EINVAL);
                 int occ = 0;
                 {

@@ -271,6 +271,33 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 #define HROW(i) hrow[(i)]
 #endif
 
+// An arrival whose lengths have not been drawn yet waits in the queue as a placeholder: prompt field 0 (a real
+// prompt has at least one token), slot of arrival, and, in the output-length field, its rank among the slot's
+// arrivals, which together are the counter of its draw.  Only the queue ring in global memory and, for a moment,
+// the window hold placeholders; convert_window draws the lengths of those inside the window, one per lane.
+__device__ __forceinline__ bool is_placeholder(uint64_t e) { return ((uint32_t)e & 0xffffu) == 0u; }
+
+__device__ __forceinline__ void convert_window(uint64_t* qwin, uint32_t wseq, uint32_t qh, int nQ, uint32_t rid,
+                                            uint32_t key0, uint32_t key1, const uint32_t* __restrict__ pool,
+                                            const uint4* __restrict__ gpool, const DevTable* tabs, int n_classes) {
+    const uint32_t lane = threadIdx.x & 31u;
+#pragma unroll 1
+    for (uint32_t half = 0; half < 2u; ++half) {
+        const uint32_t sq = wseq + 32u * half + lane;
+        const bool in = sq - qh < (uint32_t)nQ;
+        const uint64_t e = in ? qwin[sq & 63u] : 1ull;
+        if (is_placeholder(e)) {
+            uint32_t a0, a1, a2, a3;
+            philox4x32_10((uint32_t)entry_tarr(e), rid, 1u, (uint32_t)entry_o(e), key0, key1, a0, a1, a2, a3);
+            const int cls = sample_table(pool, gpool, tabs[0], a0);
+            int l, o;
+            sample_pair(pool, gpool, tabs[1 + cls], a1, tabs[1 + n_classes + cls], a2, l, o);
+            qwin[sq & 63u] = pack_entry(l, o, entry_tarr(e), cls);
+        }
+    }
+    __syncwarp();
+}
+
 // One launch advances the replicas of the groups that share one policy; a configuration with several
 // policies is run as several launches that the host issues side by side.
 // kPol: the policy, a compile-time constant: the slot loop is one long chain of short warp-uniform decisions,
@@ -287,7 +314,10 @@ __device__ __forceinline__ T& checked_ref(T* base, long long idx, long long limi
 // kBulk: the whole-prompt first-come-first-served policies (0, 1, 3, 6) first try to activate several queue heads at
 // once; the host asks for it when two or more requests arrive (and may be activated) per slot on average.  With
 // fewer the extra code only costs.
-template <int kPol, int kMinCtas, int kRec, bool kBulk>
+// kLazy: arrivals that join a long queue wait as placeholders and are drawn when the window on the queue reaches
+// them.  The host asks for it when most arrivals are dropped anyway (heavy overload) and nothing is recorded per
+// slot; elsewhere the extra code costs more than the draws it saves.
+template <int kPol, int kMinCtas, int kRec, bool kBulk, bool kLazy>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     constexpr bool kExt = kPol >= 4;
     constexpr bool kMcProfile = kPol == 6;  // MC benchmark, projection per future slot
@@ -379,6 +409,17 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         uint64_t* __restrict__ gq = reinterpret_cast<uint64_t*>(ws + p.gq_off);
         const uint32_t qmask = p.qmask;
         uint32_t wseq = qh;  // the window holds the entries with sequence numbers [wseq, wseq + 64)
+        // With kLazy, arrivals that join a long queue are not drawn at once (most are dropped when the waiting room is
+        // full, and the lengths of the others are not needed before they reach the head): they wait as placeholders
+        // and are drawn, 32 at a time, when the window reaches them.  Algorithm 1 needs the class at arrival.
+        constexpr bool kLazyOk = kLazy && kPol != 4;
+        bool q_raw = false;  // the window may hold placeholders: draw them before the head is read
+        auto q_ready = [&]() {
+            if (kLazyOk && q_raw) {
+                convert_window(qwin, wseq, qh, nQ, rid, p.key0, p.key1, p.pool, p.gpool, tabs, p.n_classes);
+                q_raw = false;
+            }
+        };
         auto q_get = [&](uint32_t seq) -> uint64_t {  // seq in [qh, qh + nQ)
             return (seq - wseq < 64u) ? qwin[seq & 63u] : gq[seq & qmask];
         };
@@ -391,6 +432,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         auto q_fill = [&](uint32_t from) {
             for (uint32_t sq = from + (uint32_t)lane; sq - wseq < 64u; sq += 32u)
                 if (sq - qh < (uint32_t)nQ) qwin[sq & 63u] = gq[sq & qmask];
+            q_raw = true;
             __syncwarp();
         };
         // one entry leaves at the head; when half of the window is used up it moves on by 32 entries
@@ -561,8 +603,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             if (lane >= L) n = 0;
             const int excl = incl - n;
             const int N = __shfl_sync(FULL, incl, L - 1);
-            // generate the N arrivals of these slots, one per lane (stream 1, index = rank within the slot)
-            for (int base = 0; base < N; base += 32) {
+            // generate the N arrivals of these slots, one per lane (stream 1, index = rank within the slot), unless
+            // they join a long queue: then those that are accepted are drawn when the window reaches them
+            const bool lazy = kLazyOk && nQ >= 96;
+            for (int base = 0; base < (lazy ? 0 : N); base += 32) {
                 const int idx = base + lane;
                 int lo = 0, hi = L - 1;
 #pragma unroll
@@ -603,10 +647,15 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     const int sp = (int)(info >> 8);  // where the slot's arrivals are staged
                     const int acc = min((int)(info & 0xffu), Qcap - nQ);
                     const uint32_t tail = qh + (uint32_t)nQ;
-                    for (int i = lane; i < acc; i += 32) {
-                        const uint64_t e = STAGE(sp + i);
-                        q_put(tail + (uint32_t)i, e);
-                        if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
+                    if (lazy) {
+                        for (int i = lane; i < acc; i += 32) q_put(tail + (uint32_t)i, pack_entry(0, i, t, 0));
+                        if (tail - wseq < 64u) q_raw = true;  // the queue has shrunk into the window meanwhile
+                    } else {
+                        for (int i = lane; i < acc; i += 32) {
+                            const uint64_t e = STAGE(sp + i);
+                            q_put(tail + (uint32_t)i, e);
+                            if ((kExt && policy == 4)) atomicAdd(&qcnt[entry_cls(e)], 1u);
+                        }
                     }
                     nQ += acc;
                     nTot += acc;
@@ -803,6 +852,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         int want = min(min(cap - a, nQ), Acap - nP);
                         if (want >= 2) {
                             want = min(want, 32);
+                            q_ready();
                             const bool in = lane < want;
                             const uint64_t e = qwin[(qh + (uint32_t)lane) & 63u];  // the first 32 queue places are in the window
                             const int l = entry_l(e);
@@ -876,7 +926,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             }
                             CADD(C_ACAP_BLOCKED, 1); status |= 1u; break;
                         }
-                        if (q_e == 0) q_e = qwin[qh & 63u];  // the head is always inside the window
+                        if (q_e == 0) {
+                            q_ready();
+                            q_e = qwin[qh & 63u];  // the head is always inside the window
+                        }
                         const int l = entry_l(q_e);
                         int g, need;
                         if (policy == 2) {

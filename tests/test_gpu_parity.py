@@ -448,3 +448,37 @@ def test_many_activations_per_slot():
         gpu = run_gpu(cfg, pieces=[333, 367])
         assert_same(cfg, gpu, ref, 700, f"many activations K={K} M={M} Acap={Acap}")
         assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 700, ref["complog"])
+
+
+def test_arrivals_drawn_when_they_reach_the_queue_head():
+    # heavy overload without per-slot outputs: the kernels that let arrivals wait undrawn in a long queue are chosen.
+    # Two-state arrivals (quiet / very busy) make the queue drain below the threshold and fill up again, so drawn and
+    # undrawn arrivals mix, late arrivals land inside the window on the queue head, evictions push requests back in
+    # front of it, bursts of up to 200 arrivals are activated in one slot, and launches are resumed in between.
+    base = wl.config5(replicas=1, T=100)
+    for i, (Qcap, M, K) in enumerate(((128, 600000, 2048), (200, 70000, 0), (256, 250000, 700))):
+        groups = (wl.Group(wl.POLICY_FLOW, b_fp=wl.b_to_fp(0.8), n_replicas=4),
+                  wl.Group(wl.POLICY_GREEDY, n_replicas=4),
+                  wl.Group(wl.POLICY_CHUNKED, chunk=512, n_replicas=3),
+                  wl.Group(wl.POLICY_ALPHA, n_replicas=3, m_admit=int(0.9 * M)),
+                  wl.Group(wl.POLICY_GREEDY, n_replicas=3, preempt_keep=1, rng_replica_base=50),
+                  wl.Group(wl.POLICY_FLOW, b_fp=wl.b_to_fp(2.5), n_replicas=3, preempt_keep=1, rng_replica_base=9))
+        arr = wl.Arrivals((wl.poisson_table(0.05), wl.poisson_table(9.0)), (1 << 25, 1 << 26))
+        cfg = base.with_(M=M, K=K, T_max=5000, Qcap=Qcap, Acap=256, seed=300 + i, arrivals=(arr,), groups=groups,
+                         trace_stride=0, complog_cap=0, hist_bins=256, hist_shift=4)
+        ref = orc.run(cfg, threads=8)
+        c = ref["counters"]
+        assert c[:, orc.CIDX["dropped"]].min() > 1000 and (i == 0 or c[:, orc.CIDX["evictions"]].sum() > 100)
+        gpu = run_gpu(cfg, pieces=[1777, 1, 3222])
+        assert_same(cfg, gpu, ref, 5000, f"undrawn arrivals {i}")
+        assert_summary_close(cfg, gpu["summary"], ref["counters"], ref["hist"], 5000, ref["complog"])
+    # short requests, a cache that takes hundreds of them, 200 arrivals in the busy slots: many activations per slot
+    burst = wl.SimConfig(
+        M=1500, K=0, T_max=600, Qcap=900, Acap=1200, seed=44, class_law=wl.constant_table(0),
+        prompt=(wl.uniform_table(1, 6),), decode=(wl.uniform_table(1, 5),),
+        arrivals=(wl.Arrivals((wl.constant_table(0), wl.constant_table(200)), (1 << 29, 1 << 30)),),
+        groups=(wl.Group(wl.POLICY_GREEDY, n_replicas=4), wl.Group(wl.POLICY_FLOW, b_fp=wl.b_to_fp(90.0), n_replicas=4)),
+        trace_stride=0, hist_bins=64, hist_shift=0, complog_cap=0)
+    ref = orc.run(burst, threads=4)
+    assert ref["counters"][:, orc.CIDX["dropped"]].min() > 0 and ref["counters"][:, orc.CIDX["admitted"]].min() > 10000
+    assert_same(burst, run_gpu(burst, pieces=[250, 350]), ref, 600, "undrawn arrivals, bursts")
