@@ -490,18 +490,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         int t = p.t0;
         const int t_end = p.t0 + p.n_steps;
 
-        // trace bookkeeping: lane (rec & 31) holds record rec until its block of 32 is flushed
+        // trace: lane k keeps the record of slot k of the current batch of draws; the batch's records are stored
+        // together when its last slot is done (one coalesced store per warp and batch)
         const int stride = (kRec == 0) ? 0 : p.trace_stride;
         const bool tracing = (kRec == 1) || (kRec == 2 && stride > 0);
-        int rec = tracing ? t / stride : 0;
-        int cd = tracing ? stride - (t % stride) : 0;
-        const int rec_lo = rec;
         int tr_u = 0, tr_q = 0;
-        // staged variant: records go to shared memory (two buffers of 32) and every full block of 32 leaves
-        // with one 256-byte bulk copy issued by lane 0, when the row's address allows it
+        // staged variant (stride 1): the batch's records go to shared memory (two buffers of 32) and leave with one
+        // bulk copy issued by lane 0 when address and size allow it (multiples of 16 bytes)
         int2* tstage = reinterpret_cast<int2*>(my + p.tstage_off);
-        const bool staged = kRec == 2 && p.tstage_off != 0 && tracing &&  // the host asks for kRec 2 with it
-                            (((reinterpret_cast<uintptr_t>(p.trace + (size_t)r * p.n_rec) - (size_t)p.rec_base * 8u) & 15u) == 0);
+        const bool staged = kRec == 2 && p.tstage_off != 0 && tracing && stride == 1;  // the host asks for kRec 2 with it
+        int tbuf = 0;
         // trow[rec] is record rec of this replica: rec_base <= rec < rec_base + n_rec
         int2* trow = (kRec != 0 && p.trace) ? p.trace + ((long long)r * p.n_rec - p.rec_base) : nullptr;
         int* hrow = p.hist ? p.hist + (size_t)r * p.hist_bins : nullptr;
@@ -1303,46 +1301,34 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 
                 // ---- record
                 maxQ = max(maxQ, nQ);
-                if (tracing && --cd == 0) {
-                    cd = stride;
-                    if (staged) {
-                        if (lane == 0) tstage[rec & 63] = make_int2(G, nQ);
-                        if ((rec & 31) == 31) {
-                            const int b0 = rec & ~31;
-                            __syncwarp();
-                            if (b0 >= rec_lo) {
-                                if (lane == 0) {
-                                    bulk_store_commit(trow + b0, tstage + (b0 & 32), 256u);
-                                    bulk_wait_read<1>();  // the other buffer (copy issued 32 records ago) is free again
-                                }
-                            } else if (b0 + lane >= rec_lo) {
-                                TROW(b0 + lane) = tstage[(b0 & 32) + lane];  // block begun by an earlier launch
-                            }
-                            __syncwarp();
+                if (kRec != 0 && lane == k) { tr_u = G; tr_q = nQ; }
+            }  // slots of the batch
+            if constexpr (kRec != 0) if (tracing) {  // the batch was the slots t - L + 1 .. t; lane k holds slot t - L + 1 + k
+                const int ts = t - L + 1 + lane;
+                if (staged) {
+                    int2* sb = tstage + 32 * tbuf;
+                    if (lane < L) sb[lane] = make_int2(tr_u, tr_q);
+                    __syncwarp();
+                    int2* dst = trow + (t - L);  // stride 1: the record of slot s has index s - 1
+                    if ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0 && (L & 1) == 0) {
+                        if (lane == 0) {
+                            bulk_store_commit(dst, sb, (uint32_t)L * 8u);
+                            bulk_wait_read<1>();  // the other buffer (copy issued a batch ago) is free again
                         }
                     } else {
-                        if (lane == (rec & 31)) { tr_u = G; tr_q = nQ; }
-                        if ((rec & 31) == 31) {
-                            const int b0 = rec & ~31;
-                            if (b0 + lane >= rec_lo) TROW(b0 + lane) = make_int2(tr_u, tr_q);
-                        }
+                        if (lane < L) TROW(ts - 1) = make_int2(tr_u, tr_q);
+                        if (lane == 0) bulk_wait_read<0>();  // no new copy: the other buffer's must have been read
                     }
-                    rec++;
+                    tbuf ^= 1;
+                    __syncwarp();
+                } else if (lane < L && (stride == 1 || ts % stride == 0)) {
+                    TROW(stride == 1 ? ts - 1 : ts / stride - 1) = make_int2(tr_u, tr_q);
                 }
-            }  // slots of the batch
+            }
             if (two_state) mstate = (smask >> (L - 1)) & 1u;
         }  // while t < t_end
 
         // ------------------------------------------------------------------ flush, final extras, spill
-        if (tracing && (rec & 31) != 0) {
-            const int b0 = rec & ~31;
-            if (staged) {
-                __syncwarp();
-                if (b0 + lane >= rec_lo && b0 + lane < rec) TROW(b0 + lane) = tstage[(b0 & 32) + lane];
-            } else if (b0 + lane >= rec_lo && b0 + lane < rec) {
-                TROW(b0 + lane) = make_int2(tr_u, tr_q);
-            }
-        }
         if (staged) {  // the staging buffers are reused by the next replica and the copies must land before the exit
             if (lane == 0) bulk_wait_all();
             __syncwarp();
