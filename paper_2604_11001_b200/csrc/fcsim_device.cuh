@@ -430,6 +430,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         // (re)load the part of the window from sequence number `from` on (all earlier queue writes of this warp
         // must be behind a __syncwarp)
         auto q_fill = [&](uint32_t from) {
+#pragma unroll 1
             for (uint32_t sq = from + (uint32_t)lane; sq - wseq < 64u; sq += 32u)
                 if (sq - qh < (uint32_t)nQ) qwin[sq & 63u] = gq[sq & qmask];
             q_raw = true;
@@ -604,6 +605,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             // generate the N arrivals of these slots, one per lane (stream 1, index = rank within the slot), unless
             // they join a long queue: then those that are accepted are drawn when the window reaches them
             const bool lazy = kLazyOk && nQ >= 96;
+#pragma unroll 1
             for (int base = 0; base < (lazy ? 0 : N); base += 32) {
                 const int idx = base + lane;
                 int lo = 0, hi = L - 1;
@@ -646,9 +648,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                     const int acc = min((int)(info & 0xffu), Qcap - nQ);
                     const uint32_t tail = qh + (uint32_t)nQ;
                     if (lazy) {
+#pragma unroll 1
                         for (int i = lane; i < acc; i += 32) q_put(tail + (uint32_t)i, pack_entry(0, i, t, 0));
                         if (tail - wseq < 64u) q_raw = true;  // the queue has shrunk into the window meanwhile
                     } else {
+#pragma unroll 1
                         for (int i = lane; i < acc; i += 32) {
                             const uint64_t e = STAGE(sp + i);
                             q_put(tail + (uint32_t)i, e);
@@ -668,6 +672,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 // ---- chunked policy: continuing prefills first, in activation order
                 if (policy == 2 && n_pref > 0) {
                     int first_left = -1;
+#pragma unroll 1
                     for (int base = pf_lo & ~31; base < nP; base += 32) {
                         const int i = base + lane;
                         uint32_t sw = 0;
@@ -864,6 +869,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 // other (each is booked on the projection before the next is tested); the first
                                 // refusal ends the run
                                 int pass = 0;
+#pragma unroll 1
                                 for (; pass < n; ++pass) {
                                     const uint64_t ec = __shfl_sync(FULL, e, pass);
                                     const int op_c = grp.mc_worst != 0 ? (tabs[1 + p.n_classes + entry_cls(ec)].vmin +
@@ -871,11 +877,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                                                        : entry_o(ec);
                                     const int a_c = entry_l(ec) - t + 1;
                                     bool over = false;
+#pragma unroll 1
                                     for (int base = 0; base < op_c; base += 32) {
                                         const int tau = t + base + lane;
                                         over |= (base + lane < op_c) && (vproj[(uint32_t)tau & p.prof_mask] + a_c + tau > M);
                                     }
                                     if (__any_sync(FULL, over)) break;
+#pragma unroll 1
                                     for (int base = 0; base < op_c; base += 32) {
                                         const int tau = t + base + lane;
                                         if (base + lane < op_c) vproj[(uint32_t)tau & p.prof_mask] += a_c + tau;
@@ -915,6 +923,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             }
                         }
                     }
+#pragma unroll 1
                     while (a < cap && nQ > 0) {
                         if (nP == Acap) {
                             if (nD > 0) {  // storage, not the model's bound: make room
@@ -955,11 +964,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                                                : entry_o(eh);
                             const int a_h = l - t + 1;
                             bool over = false;
+#pragma unroll 1
                             for (int base = 0; base < op_h; base += 32) {
                                 const int tau = t + base + lane;
                                 over |= (base + lane < op_h) && (vproj[(uint32_t)tau & p.prof_mask] + a_h + tau > M);
                             }
                             if (__any_sync(FULL, over)) { CADD(C_GATE_BLOCKED, 1); break; }
+#pragma unroll 1
                             for (int base = 0; base < op_h; base += 32) {
                                 const int tau = t + base + lane;
                                 if (base + lane < op_h) vproj[(uint32_t)tau & p.prof_mask] += a_h + tau;
@@ -1115,6 +1126,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         cmin = kNoFin;
                         next_fin = kNoFin;
                     }
+#pragma unroll 1
                     while (policy != 3 && G > M && nP > nD) {
                         int i = nP - 1;
                         uint32_t sw = STATE(WA(shead + i));
@@ -1124,6 +1136,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             // is still needed for its statistics); it is evicted from the top place below
                             const uint32_t sw_top = sw;
                             int found = -1;
+#pragma unroll 1
                             for (int top = nP; found < 0 && top > 0; top -= 32) {
                                 const int idx = top - 32 + lane;
                                 const uint32_t w = (idx >= 0) ? STATE(WA(shead + idx)) : kDead;
@@ -1207,11 +1220,13 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         npend = 0;
                     };
                     uint32_t due = __ballot_sync(FULL, cmin == (uint32_t)t);
+#pragma unroll 1
                     while (due) {
                         const int c = __ffs(due) - 1;
                         due &= due - 1;
                         uint32_t gmin = kNoFin;  // new minimum of lane c's stretch
                         const int stop = min(nP, (c + 1) << bsh);
+#pragma unroll 1
                         for (int base = c << bsh; base < stop; base += 32) {
                             const int i = base + lane;
                             const uint32_t sw = (i < nP) ? STATE(WA(shead + i)) : kDead;
@@ -1236,6 +1251,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                     // f_c = t + (longest output of its class - o) leaves the projected usage of the
                                     // slots t+1 .. f_c, where it was booked with a_c + tau, a_c = l + o - t
                                     uint32_t mm = m;
+#pragma unroll 1
                                     while (mm) {
                                         const int src = __ffs(mm) - 1;
                                         mm &= mm - 1;
@@ -1243,6 +1259,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                         const DevTable dc = tabs[1 + p.n_classes + entry_cls(ec)];
                                         const int extra = dc.vmin + (int)dc.n - 1 - entry_o(ec);  // slots it leaves early
                                         const int a_c = entry_l(ec) + entry_o(ec) - t;
+#pragma unroll 1
                                         for (int base = 0; base < extra; base += 32) {
                                             const int tau = t + 1 + base + lane;
                                             if (base + lane < extra) vproj[(uint32_t)tau & p.prof_mask] -= a_c + tau;
