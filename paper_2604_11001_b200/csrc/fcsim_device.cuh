@@ -232,6 +232,14 @@ __device__ __forceinline__ long long warp_sum64(long long v) {
     return v;
 }
 
+// A value that every lane of the warp holds, handed to the compiler as such: the result of a warp-wide reduction
+// is uniform by construction, so conditions and loop bounds computed from it need no reconvergence bookkeeping.
+__device__ __forceinline__ uint32_t uni(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
+__device__ __forceinline__ int uni(int v) { return (int)__reduce_max_sync(0xffffffffu, (uint32_t)v); }
+__device__ __forceinline__ uint64_t uni(uint64_t v) {
+    return ((uint64_t)__reduce_max_sync(0xffffffffu, (uint32_t)(v >> 32)) << 32) | __reduce_max_sync(0xffffffffu, (uint32_t)v);
+}
+
 __device__ __forceinline__ uint64_t pack_entry(int l, int o, int t_arr, int cls) {
     return (uint64_t)(uint32_t)(l | (o << 16)) | ((uint64_t)(uint32_t)(t_arr | (cls << 24)) << 32);
 }
@@ -360,7 +368,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         // ------------------------------------------------------------------ next replica
         unsigned int wi = 0;  // work item: the wi-th replica of this policy
         if (lane == 0) wi = atomicAdd(p.work_counter, 1u);
-        wi = __shfl_sync(FULL, wi, 0);
+        wi = uni(wi);  // lane 0 holds it, the others zero
         if (wi >= (unsigned)p.n_work) break;
 
         int gi = 0;
@@ -370,15 +378,19 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                 const int mid = (lo + hi + 1) >> 1;
                 if (p.groups[mid].wfirst <= (int)wi) lo = mid; else hi = mid - 1;
             }
-            gi = lo;
+            gi = uni(lo);
         }
-        const DevGroup grp = p.groups[gi];
+        DevGroup grp = p.groups[gi];
+        grp.b_fp = uni(grp.b_fp); grp.chunk = uni(grp.chunk); grp.arrivals_id = uni(grp.arrivals_id);
+        grp.rng_base = uni(grp.rng_base); grp.first = uni(grp.first); grp.admit_limit = uni(grp.admit_limit);
+        grp.bclass_off = uni(grp.bclass_off); grp.mc_worst = uni(grp.mc_worst); grp.keep = uni(grp.keep);
+        grp.wfirst = uni(grp.wfirst);
         const unsigned int r = (unsigned)grp.first + (wi - (unsigned)grp.wfirst);  // the replica's index
         const DevArrivals* arrp = p.arrivals + grp.arrivals_id;
         const DevTable cnt0 = arrp->count[0];
         const DevTable cnt1 = arrp->count[1];
         const uint32_t thr0 = arrp->thr[0], thr1 = arrp->thr[1];
-        const bool two_state = arrp->n_states == 2;
+        const bool two_state = uni(arrp->n_states) == 2u;
         const uint32_t rid = grp.rng_base + (r - (unsigned)grp.first);
         constexpr int policy = kPol;
         const int chunk = grp.chunk;
@@ -388,18 +400,19 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         unsigned char* ws = p.workspace + (size_t)r * p.ws_stride;
         uint32_t* hdr = reinterpret_cast<uint32_t*>(ws);
         const uint32_t hw = (lane < kHeaderWords) ? hdr[lane] : 0u;
-        uint32_t qh = __shfl_sync(FULL, hw, 0);       // sequence number of the queue head (ring place = qh & qmask)
-        int shead = (int)__shfl_sync(FULL, hw, 1);    // ring position of the oldest active entry
-        int nP = (int)__shfl_sync(FULL, hw, 2);       // entries in the active range, completed ones included
-        int nQ = (int)__shfl_sync(FULL, hw, 3);
-        int U = (int)__shfl_sync(FULL, hw, 4);        // usage carried out of the last slot, completions released
-        int Ndec = (int)__shfl_sync(FULL, hw, 5);     // active requests whose prompt is fully in the cache
-        uint32_t next_fin = ~__shfl_sync(FULL, hw, 6);  // stored complemented so that zeroed memory means "none"
-        int n_pref = (int)__shfl_sync(FULL, hw, 7);   // active requests still prefilling
-        int pf_lo = (int)__shfl_sync(FULL, hw, 8);    // lower bound on the index of the oldest of those
-        uint32_t mstate = __shfl_sync(FULL, hw, 9);
-        uint32_t status = __shfl_sync(FULL, hw, 10);
-        int nD = (int)__shfl_sync(FULL, hw, 11);      // completed entries still inside the active range
+        auto hword = [&](int j) { return uni(lane == j ? hw : 0u); };
+        uint32_t qh = hword(0);                 // sequence number of the queue head (ring place = qh & qmask)
+        int shead = (int)hword(1);              // ring position of the oldest active entry
+        int nP = (int)hword(2);                 // entries in the active range, completed ones included
+        int nQ = (int)hword(3);
+        int U = (int)hword(4);                  // usage carried out of the last slot, completions released
+        int Ndec = (int)hword(5);               // active requests whose prompt is fully in the cache
+        uint32_t next_fin = ~hword(6);          // stored complemented so that zeroed memory means "none"
+        int n_pref = (int)hword(7);             // active requests still prefilling
+        int pf_lo = (int)hword(8);              // lower bound on the index of the oldest of those
+        uint32_t mstate = hword(9);
+        uint32_t status = hword(10);
+        int nD = (int)hword(11);                // completed entries still inside the active range
         {
             const uint4* src = reinterpret_cast<const uint4*>(ws + kHeaderWords * 4);
             uint4* dst = reinterpret_cast<uint4*>(my);
@@ -471,7 +484,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
         uint32_t sumN = 0, tokgen = 0, arrived = 0, accepted = 0;
         int maxU = 0, maxQ = 0;
         int nTot = nP - nD + nQ;  // requests in the system: changes only when requests arrive or complete
-        int n_logged = (int)__shfl_sync(FULL, (int)cnt, C_N_LOGGED);
+        int n_logged = uni(lane == C_N_LOGGED ? (int)cnt : 0);
         uint64_t q_e = 0;  // the queue head's entry when known, else 0 (saves shared-memory reads in blocked slots)
         // Whole-prompt policies: once the headroom gate has refused the queue head, it keeps refusing it until
         // memory is released (a completion or an eviction): the usage only grows and the head does not change.
@@ -601,7 +614,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             L = min(L, __popc(__ballot_sync(FULL, incl <= S)));  // staged arrivals must fit; n <= S so L >= 1
             if (lane >= L) n = 0;
             const int excl = incl - n;
-            const int N = __shfl_sync(FULL, incl, L - 1);
+            const int N = uni(lane == L - 1 ? incl : 0);
             // generate the N arrivals of these slots, one per lane (stream 1, index = rank within the slot), unless
             // they join a long queue: then those that are accepted are drawn when the window reaches them
             const bool lazy = kLazyOk && nQ >= 96;
@@ -643,7 +656,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 
                 // ---- arrivals join the queue tail; a full waiting room drops the rest
                 if (((nzmask >> k) & 1u) && nQ < Qcap) {
-                    const uint32_t info = __shfl_sync(FULL, packed, k);
+                    const uint32_t info = uni(lane == k ? packed : 0u);
                     const int sp = (int)(info >> 8);  // where the slot's arrivals are staged
                     const int acc = min((int)(info & 0xffu), Qcap - nQ);
                     const uint32_t tail = qh + (uint32_t)nQ;
@@ -905,7 +918,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 if (lane == c0) cmin = min(cmin, m0);
                                 if (lane == c0 + 1) cmin = min(cmin, m1);
                                 next_fin = min(next_fin, min(m0, m1));
-                                const int tot = __shfl_sync(FULL, pre, n - 1);
+                                const int tot = uni(lane == n - 1 ? pre : 0);
                                 G += tot;
                                 if (!kinf) R = max(0, R - (tot - n));
                                 Ndec += n;
@@ -935,7 +948,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                         }
                         if (q_e == 0) {
                             q_ready();
-                            q_e = qwin[qh & 63u];  // the head is always inside the window
+                            q_e = uni(qwin[qh & 63u]);  // the head is always inside the window
                         }
                         const int l = entry_l(q_e);
                         int g, need;
@@ -1129,7 +1142,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 #pragma unroll 1
                     while (policy != 3 && G > M && nP > nD) {
                         int i = nP - 1;
-                        uint32_t sw = STATE(WA(shead + i));
+                        uint32_t sw = uni(STATE(WA(shead + i)));
                         if (is_dead(sw)) {
                             // completed entries lie on top of the newest live one: find it (backwards, 32 at a
                             // time), and let it change places with the completed entry at the top (whose record
@@ -1144,7 +1157,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                                 if (m) found = top - 1 - __clz(m);
                             }
                             i = found;
-                            sw = STATE(WA(shead + i));
+                            sw = uni(STATE(WA(shead + i)));
                             const uint64_t moved = RING(WA(shead + i));
                             const uint64_t top_e = RING(WA(shead + nP - 1));
                             __syncwarp();
@@ -1155,7 +1168,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
                             }
                             __syncwarp();
                         }
-                        uint64_t e = RING(WA(shead + nP - 1));
+                        uint64_t e = uni(RING(WA(shead + nP - 1)));
                         if (sw & kPrefillBit) {
                             G -= (int)(sw & ~kPrefillBit);
                             n_pref--;
