@@ -469,8 +469,12 @@ template <int kPol, int kCtas>
 static step_kernel_t step_kernel_for(int rec, bool bulk, bool lazy) {
     constexpr bool kFifo = kPol <= 1 || kPol == 3 || kPol == 6;
     constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 .. 6 uninstantiated
-    // lazily drawn arrivals: only the forms that record nothing per slot, without the several-heads step
-    if (kPol <= 3 && lazy && !bulk && rec == 0) return fcsim_step_kernel<kP, kCtas, 0, false, kPol <= 3>;
+    // lazily drawn arrivals: without the several-heads step
+    if (kPol <= 3 && lazy && !bulk) {
+        if (rec == 2) return fcsim_step_kernel<kP, kCtas, 2, false, kPol <= 3>;
+        if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, false, kPol <= 3>;
+        return fcsim_step_kernel<kP, kCtas, 0, false, kPol <= 3>;
+    }
     if (kFifo && bulk) {
         if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, kFifo, false>;
         if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, kFifo, false>;
