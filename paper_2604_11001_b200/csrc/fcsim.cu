@@ -33,6 +33,9 @@ struct Layout {
     size_t tstage_off;                          // trace staging buffers, 0 = unused
     size_t state_bytes;                         // ring + state words (+ projection words) saved between launches
     int has_v;
+    int min_S;                                  // staging places a slot's arrivals need at most (the largest count)
+    int qcnt_classes;                           // classes with a per-class queue count (Algorithm 1 groups), else 0
+    int staged_trace;                           // 1 = trace staging buffers (trace_bulk)
     uint32_t prof_mask;                         // MC benchmark: H - 1 when the projection is kept per future slot, else 0
     int warps_per_block;
     int n_rec;
@@ -93,6 +96,26 @@ double capacity_rate(const fcsim_config* c) {
         prev = cum;
     }
     return ew > 0.0 ? (double)c->M / ew : 0.0;
+}
+
+// A warp's shared memory for S staging places: saved state, staged arrivals, queue window (64 entries), per-class
+// queue counts (Algorithm 1), and the optional trace staging (fcsim_config::trace_bulk = 1: 2 x 32 records of 8
+// bytes, each batch leaving with one bulk copy; off by default: measured slower than keeping the records in
+// registers, and the extra shared memory costs a CTA).
+void set_staging(Layout* L, int S) {
+    L->S = S;
+    L->qwin_off = L->state_bytes + (size_t)S * 8;
+    L->qcnt_off = L->qwin_off + 64 * 8;
+    L->smem_per_warp = L->qcnt_off + (L->qcnt_classes ? align_up((size_t)L->qcnt_classes * 4, 16) : 0);
+    if (!L->qcnt_classes) L->qcnt_off = 0;
+    L->tstage_off = 0;
+    if (L->staged_trace) {
+        L->tstage_off = L->smem_per_warp;
+        L->smem_per_warp += 512;
+    }
+    int w = kWarpsPerBlock;
+    while (w > 1 && (size_t)w * L->smem_per_warp > kSmemBudget) w >>= 1;
+    L->warps_per_block = w;
 }
 
 // Validates the description and derives the storage layout.  Returns an FCSIM_* code.
@@ -171,24 +194,12 @@ int plan(const fcsim_config* c, Layout* L) {
     // workspace record of a replica: 16 header words, the saved shared-memory state, the queue ring
     L->gq_off = kHeaderWords * 4 + L->state_bytes;
     L->ws_stride = L->gq_off + (size_t)L->QC * 8;
-    // a warp's shared memory: saved state, staged arrivals, queue window (64 entries), per-class queue counts
-    L->qwin_off = L->state_bytes + (size_t)L->S * 8;
-    L->qcnt_off = L->qwin_off + 64 * 8;
-    L->smem_per_warp = L->qcnt_off + (any_classflow ? align_up((size_t)c->n_classes * 4, 16) : 0);
-    if (!any_classflow) L->qcnt_off = 0;
-    // Optional trace staging (fcsim_config::trace_bulk = 1): 2 x 32 records of 8 bytes in shared memory,
-    // each full block leaving with one 256-byte bulk copy.  Off by default: measured slower than keeping
-    // the records in registers (the stream is 8 bytes per slot, and the extra shared memory costs a CTA).
-    L->tstage_off = 0;
     if (c->trace_bulk < 0 || c->trace_bulk > 1) return FCSIM_EINVAL;
-    if (c->trace_stride > 0 && c->trace_bulk == 1) {
-        L->tstage_off = L->smem_per_warp;
-        L->smem_per_warp += 512;
-    }
+    L->min_S = (int)align_up((size_t)std::max(32, max_count), 2);
+    L->qcnt_classes = any_classflow ? c->n_classes : 0;
+    L->staged_trace = (c->trace_stride > 0 && c->trace_bulk == 1) ? 1 : 0;
+    set_staging(L, L->S);
     if (L->smem_per_warp > kSmemBudget) return FCSIM_ECAP;
-    int w = kWarpsPerBlock;
-    while (w > 1 && (size_t)w * L->smem_per_warp > kSmemBudget) w >>= 1;
-    L->warps_per_block = w;
     L->n_rec = c->trace_stride > 0 ? c->T_max / c->trace_stride : 0;
     L->R = R;
     return FCSIM_OK;
@@ -487,6 +498,7 @@ static step_kernel_t step_kernel_for(int rec, bool bulk, bool lazy) {
 template <int kPol>
 static step_kernel_t step_kernel_for(int ctas, int rec, bool bulk, bool lazy) {
     switch (ctas) {
+        case 8: return step_kernel_for<kPol, 8>(rec, bulk, lazy);
         case 5: return step_kernel_for<kPol, 5>(rec, bulk, lazy);
         case 6: return step_kernel_for<kPol, 6>(rec, bulk, lazy);
         default: return step_kernel_for<kPol, 7>(rec, bulk, lazy);
@@ -514,6 +526,7 @@ struct PolicyLaunch {
     int n_work = 0;               // replicas
     bool bulk = false;            // two or more requests arrive, and may be activated, per slot on average
     bool lazy = false;            // at least twice as many requests arrive as the cache can serve: most are dropped
+    double busiest = 0.0;         // requests that arrive per slot, the largest over the policy's groups
     int warps_per_block = 0, blocks_per_sm = 0, grid = 0;
     size_t smem_block = 0, tabcache_off = 0;
     cudaStream_t side = nullptr;  // null: the caller's stream
@@ -701,6 +714,7 @@ static int upload_tables(fcsim* h, const fcsim_config* c) {
         pl.bulk = std::min(most, cap_rate) >= 2.0;
         // heavy overload with a waiting room long enough to hide the head: arrivals are drawn when they get there
         pl.lazy = busiest >= 2.0 * cap_rate && c->Qcap >= 128;
+        pl.busiest = busiest;
         pl.pg_cnt = (int)pgrps.size() - pl.pg_off;
         if (pl.pg_cnt > 0) h->launches.push_back(pl);
     }
@@ -803,11 +817,14 @@ static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_
     }
     if (rc != FCSIM_OK) return fail(rc);
 
-    // Launch shape, per policy kernel: warps per CTA (1 .. 4) and register allocation (<= 96 registers, or <= 80)
-    // are chosen for the largest number of resident warps per SM, as the occupancy calculator reports it for this
-    // device; ties go to the roomier register allocation, then to the larger CTA.  A warp's slice of shared memory
-    // is fixed by the configuration, so small slices end up register-bound (6 CTAs of 4 warps at 80 registers)
-    // and large ones shared-memory-bound, where smaller CTAs waste less of the SM's 228 KB.
+    // Launch shape, per policy kernel: warps per CTA (1 .. 4) and register allocation (builds for 5, 6, 7 and 8
+    // resident CTAs: <= 96, 80, 72, 64 registers) are chosen for the largest number of resident warps per SM, as the
+    // occupancy calculator reports it for this device; ties go to the roomier register allocation, then to the
+    // larger CTA.  Small slices of shared memory end up register-bound, large ones shared-memory-bound, where
+    // smaller CTAs waste less of the SM's 228 KB.  The staging area for generated arrivals is the one part of a
+    // warp's slice that the library may size: the shapes are worked out for the roomy one (128 places: a batch of 32
+    // slots rarely has to be cut short) and for the smallest one (the largest arrival count of a slot, at least
+    // 32), and the small one is taken when it lets more warps reside (Acap = 512: 8 CTAs of 4 warps instead of 7).
     const bool ext = L.qcnt_off || L.has_v;
     // what is recorded per slot is a compile-time property of the kernels of the common policies
     const int rec = (ext || cfg->complog_cap > 0 || L.tstage_off != 0) ? 2 : (L.n_rec > 0 ? 1 : 0);
@@ -815,8 +832,9 @@ static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_
     const size_t sm_bytes = (size_t)prop.sharedMemPerMultiprocessor;
     auto ctas_by_smem = [&](size_t b) { return sm_bytes / (align_up(b, 1024) + 1024); };
     size_t most_work = 0;
-    for (size_t li = 0; li < h->launches.size(); ++li) {
-        PolicyLaunch& pl = h->launches[li];
+    auto shape = [&](const Layout& L, std::vector<PolicyLaunch>& launches) -> int {
+    for (size_t li = 0; li < launches.size(); ++li) {
+        PolicyLaunch& pl = launches[li];
         int best_warps = 0;
         for (int w = L.warps_per_block; w >= 1; --w) {
             size_t block = (size_t)w * L.smem_per_warp, tab = 0;
@@ -827,17 +845,17 @@ static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_
                 tab = block;
                 block += tab_extra;
             }
-            for (int ctas = 5; ctas <= 7; ++ctas) {
+            for (int ctas = 5; ctas <= 8; ++ctas) {
                 step_kernel_t k = pick_step_kernel(pl.policy == FCSIM_POLICY_MC && L.prof_mask ? 6 : pl.policy, ctas, rec,
                                                    pl.bulk, pl.lazy);
-                if (!k) return fail(FCSIM_EINVAL);
+                if (!k) return FCSIM_EINVAL;
                 int occ = 0;
                 {
                     std::lock_guard<std::mutex> lock(g_kernel_attr_mutex);
                     e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block);
                     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, w * 32, block);
                 }
-                if (e != cudaSuccess) { h->last_cuda = (int)e; return fail(FCSIM_ECUDA); }
+                if (e != cudaSuccess) { h->last_cuda = (int)e; return FCSIM_ECUDA; }
                 if (occ * w > best_warps) {
                     best_warps = occ * w;
                     pl.kernel = k;
@@ -848,10 +866,37 @@ static int create_handle(const fcsim_config* cfg, const fcsim_buffers* b, fcsim_
                 }
             }
         }
-        if (best_warps < 1) return fail(FCSIM_ECAP);
+        if (best_warps < 1) return FCSIM_ECAP;
         const long long want = ((long long)pl.n_work + pl.warps_per_block - 1) / pl.warps_per_block;
         pl.grid = (int)std::max<long long>(1, std::min<long long>((long long)h->sm_count * pl.blocks_per_sm, want));
         if ((size_t)pl.n_work > most_work) { most_work = (size_t)pl.n_work; h->main_launch = (int)li; }
+    }
+    return FCSIM_OK;
+    };
+    {
+        std::vector<PolicyLaunch> roomy = h->launches, tight = h->launches;
+        Layout Lt = L;
+        set_staging(&Lt, L.min_S);
+        rc = shape(L, roomy);
+        if (rc == FCSIM_OK && Lt.S < L.S) {
+            most_work = 0;
+            rc = shape(Lt, tight);
+        }
+        if (rc != FCSIM_OK) return fail(rc);
+        // More resident warps pay when they shorten the run by whole waves of replicas (the warps take replicas from
+        // a common queue: with the same number of waves every warp is merely slower), and a small staging area only
+        // where a batch of 32 slots rarely overflows it (or is not staged at all: arrivals drawn at the queue head).
+        const int m = h->main_launch;
+        const long long wr = (long long)roomy[m].blocks_per_sm * roomy[m].warps_per_block * h->sm_count;
+        const long long wt = (long long)tight[m].blocks_per_sm * tight[m].warps_per_block * h->sm_count;
+        const bool fits = tight[m].lazy || tight[m].busiest * 32.0 <= 2.0 * Lt.S;
+        if (Lt.S < L.S && fits && wt > wr && (L.R + wt - 1) / wt < (L.R + wr - 1) / wr) {
+            h->launches = tight;
+            L = Lt;
+            h->L = Lt;
+        } else {
+            h->launches = roomy;
+        }
     }
     // several policies: their launches run side by side (the first on the caller's stream, the others on streams
     // of the handle, forked from and joined to the caller's stream by events), so that no SM idles while the last

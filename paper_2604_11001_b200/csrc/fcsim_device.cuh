@@ -611,13 +611,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
             }
             if (lane >= L) n = 0;
             int incl = warp_incl_scan(n, lane);
-            L = min(L, __popc(__ballot_sync(FULL, incl <= S)));  // staged arrivals must fit; n <= S so L >= 1
+            // arrivals that join a long queue are not generated now (see below): nothing is staged
+            const bool lazy = kLazyOk && nQ >= 96;
+            if (!lazy) L = min(L, __popc(__ballot_sync(FULL, incl <= S)));  // staged arrivals must fit; n <= S so L >= 1
             if (lane >= L) n = 0;
             const int excl = incl - n;
             const int N = uni(lane == L - 1 ? incl : 0);
             // generate the N arrivals of these slots, one per lane (stream 1, index = rank within the slot), unless
             // they join a long queue: then those that are accepted are drawn when the window reaches them
-            const bool lazy = kLazyOk && nQ >= 96;
 #pragma unroll 1
             for (int base = 0; base < (lazy ? 0 : N); base += 32) {
                 const int idx = base + lane;
