@@ -37,7 +37,8 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
 
 def _compile(lib: str, verbose: bool, extra) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    # -split-compile 0: the kernels (one instantiation per policy and variant) are optimised on all host cores
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-split-compile", "0",
            "-Xcompiler", "-fPIC,-Wall", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
