@@ -465,54 +465,23 @@ __global__ void __launch_bounds__(256) latency_select_kernel(const unsigned long
 
 }  // namespace
 
-typedef void (*step_kernel_t)(const Params);
-
 // The opt-in shared-memory limit is a property of a kernel, shared by every handle of the process: setting it
 // and using it (occupancy query, launch) happen under this lock, so that handles driven from different threads do
 // not change it between another handle's two steps.
 static std::mutex g_kernel_attr_mutex;
 
-// The step kernel compiled for one policy, for a register allocation that lets 7, 6 or 5 CTAs reside on an SM, for
-// what is recorded per slot (0 nothing, 1 trace only, 2 decided at run time; Algorithm 1 and the MC benchmark
-// exist in the run-time form only) and, for the whole-prompt first-come-first-served policies, with or without the
-// activation of several queue heads at once.
-template <int kPol, int kCtas>
-static step_kernel_t step_kernel_for(int rec, bool bulk, bool lazy) {
-    constexpr bool kFifo = kPol <= 1 || kPol == 3 || kPol == 6;
-    constexpr int kP = kPol >= 4 ? 0 : kPol;  // keeps the specialised forms of policies 4 .. 6 uninstantiated
-    // lazily drawn arrivals: without the several-heads step
-    if (kPol <= 3 && lazy && !bulk) {
-        if (rec == 2) return fcsim_step_kernel<kP, kCtas, 2, false, kPol <= 3>;
-        if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, false, kPol <= 3>;
-        return fcsim_step_kernel<kP, kCtas, 0, false, kPol <= 3>;
-    }
-    if (kFifo && bulk) {
-        if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, kFifo, false>;
-        if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, kFifo, false>;
-        return fcsim_step_kernel<kP, kCtas, 0, kFifo, false>;
-    }
-    if (kPol >= 4 || rec == 2) return fcsim_step_kernel<kPol, kCtas, 2, false, false>;
-    if (rec == 1) return fcsim_step_kernel<kP, kCtas, 1, false, false>;
-    return fcsim_step_kernel<kP, kCtas, 0, false, false>;
-}
-template <int kPol>
-static step_kernel_t step_kernel_for(int ctas, int rec, bool bulk, bool lazy) {
-    switch (ctas) {
-        case 8: return step_kernel_for<kPol, 8>(rec, bulk, lazy);
-        case 5: return step_kernel_for<kPol, 5>(rec, bulk, lazy);
-        case 6: return step_kernel_for<kPol, 6>(rec, bulk, lazy);
-        default: return step_kernel_for<kPol, 7>(rec, bulk, lazy);
-    }
-}
+// The step kernel of one policy (6: the MC benchmark with its projection per future slot) for a register
+// allocation that lets `ctas` CTAs reside on an SM and for a variant; each policy's kernels are an object of their
+// own (fcsim_step_kernels.cu).
 static step_kernel_t pick_step_kernel(int policy, int ctas, int rec, bool bulk, bool lazy) {
     switch (policy) {
-        case FCSIM_POLICY_FLOW: return step_kernel_for<0>(ctas, rec, bulk, lazy);
-        case FCSIM_POLICY_GREEDY: return step_kernel_for<1>(ctas, rec, bulk, lazy);
-        case FCSIM_POLICY_CHUNKED: return step_kernel_for<2>(ctas, rec, bulk, lazy);
-        case FCSIM_POLICY_ALPHA: return step_kernel_for<3>(ctas, rec, bulk, lazy);
-        case FCSIM_POLICY_CLASSFLOW: return step_kernel_for<4>(ctas, rec, bulk, lazy);
-        case FCSIM_POLICY_MC: return step_kernel_for<5>(ctas, rec, bulk, lazy);
-        case 6: return step_kernel_for<6>(ctas, rec, bulk, lazy);  // the MC benchmark with its projection per future slot
+        case FCSIM_POLICY_FLOW: return step_kernel_of_policy_0(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_GREEDY: return step_kernel_of_policy_1(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_CHUNKED: return step_kernel_of_policy_2(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_ALPHA: return step_kernel_of_policy_3(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_CLASSFLOW: return step_kernel_of_policy_4(ctas, rec, bulk, lazy);
+        case FCSIM_POLICY_MC: return step_kernel_of_policy_5(ctas, rec, bulk, lazy);
+        case 6: return step_kernel_of_policy_6(ctas, rec, bulk, lazy);
         default: return nullptr;
     }
 }

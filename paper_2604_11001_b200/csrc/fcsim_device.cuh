@@ -232,6 +232,14 @@ __device__ __forceinline__ long long warp_sum64(long long v) {
     return v;
 }
 
+// A value computed ONCE: it passes through a register move that the compiler will not repeat.  The lane and
+// warp numbers and the warp's offsets in shared memory are cheap to derive from the thread index, so cheap that
+// the compiler otherwise derives them again at most of their hundreds of uses instead of keeping them, which
+// costs more than a tenth of all executed instructions.  Only integers take this route: a pointer would lose
+// its address space on the way.
+__device__ __forceinline__ uint32_t once(uint32_t v) { uint32_t r; asm("mov.b32 %0, %1;" : "=r"(r) : "r"(v)); return r; }
+__device__ __forceinline__ int once(int v) { int r; asm("mov.b32 %0, %1;" : "=r"(r) : "r"(v)); return r; }
+
 // A value that every lane of the warp holds, handed to the compiler as such: the result of a warp-wide reduction
 // is uniform by construction, so conditions and loop bounds computed from it need no reconvergence bookkeeping.
 __device__ __forceinline__ uint32_t uni(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
@@ -317,14 +325,14 @@ __device__ __forceinline__ void convert_window(uint64_t* qwin, uint32_t wseq, ui
 // benchmark (policy 5) use extra per-warp state (class counts, projection words).
 // kPol 6 is the MC benchmark again, with its projection kept per future slot instead of per active entry
 // (the host picks it when the longest output length is short next to the active set's storage).
-// kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80).  The host
-// asks the occupancy calculator about both.
+// kMinCtas: resident CTAs per SM the register allocation must allow (5: <= 96 registers, 6: <= 80, 7: <= 72,
+// 8: <= 64).  The host asks the occupancy calculator about all of them.
 // kBulk: the whole-prompt first-come-first-served policies (0, 1, 3, 6) first try to activate several queue heads at
 // once; the host asks for it when two or more requests arrive (and may be activated) per slot on average.  With
 // fewer the extra code only costs.
 // kLazy: arrivals that join a long queue wait as placeholders and are drawn when the window on the queue reaches
-// them.  The host asks for it when most arrivals are dropped anyway (heavy overload) and nothing is recorded per
-// slot; elsewhere the extra code costs more than the draws it saves.
+// them.  The host asks for it when most arrivals are dropped anyway (heavy overload); elsewhere the extra code
+// costs more than the draws it saves.
 template <int kPol, int kMinCtas, int kRec, bool kBulk, bool kLazy>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kernel(const Params p) {
     constexpr bool kExt = kPol >= 4;
@@ -344,17 +352,20 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
     }
     __syncthreads();
     const DevTable* __restrict__ tabs = tab_shared ? s_tables : p.tables;
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    unsigned char* my = smem_raw + (size_t)warp * p.smem_per_warp;
+    const int lane = once((int)(threadIdx.x & 31));
+    const int warp = once((int)(threadIdx.x >> 5));
+    // the warp's slice of shared memory and the areas in it, each as an offset that is computed once
+    const uint32_t my_off = (uint32_t)warp * p.smem_per_warp;
+    unsigned char* my = smem_raw + once(my_off);
     uint64_t* ring = reinterpret_cast<uint64_t*>(my);
-    uint32_t* state = reinterpret_cast<uint32_t*>(my + (size_t)p.Apad * 8);
+    uint32_t* state = reinterpret_cast<uint32_t*>(smem_raw + once(my_off + (uint32_t)p.Apad * 8u));
     // MC benchmark: vproj[k] = memory usage projected for the last slot of active entry k (same ring as state)
-    int* vproj = reinterpret_cast<int*>(state + p.Apad);
+    int* vproj = reinterpret_cast<int*>(smem_raw + once(my_off + (uint32_t)p.Apad * 12u));
     const int state_bytes = (int)p.state_bytes;  // multiple of 16 (host guarantees)
-    uint64_t* stage = reinterpret_cast<uint64_t*>(my + state_bytes);
-    uint32_t* qcnt = reinterpret_cast<uint32_t*>(my + p.qcnt_off);  // waiting requests per class (Algorithm 1 only)
-    uint64_t* qwin = reinterpret_cast<uint64_t*>(my + p.qwin_off);   // window on the queue head (64 entries)
+    uint64_t* stage = reinterpret_cast<uint64_t*>(smem_raw + once(my_off + (uint32_t)state_bytes));
+    // waiting requests per class (Algorithm 1 only)
+    uint32_t* qcnt = reinterpret_cast<uint32_t*>(smem_raw + once(my_off + p.qcnt_off));
+    uint64_t* qwin = reinterpret_cast<uint64_t*>(smem_raw + once(my_off + p.qwin_off));  // window on the queue head (64 entries)
 
     const int Acap = p.Acap, Qcap = p.Qcap, M = p.M, K = p.K, S = p.S;
     const bool kinf = (K == 0);
@@ -1433,5 +1444,16 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, kMinCtas) fcsim_step_kern
 #undef WA
     }
 }
+
+// What the host launches: one function per policy's object (fcsim_step_kernels.cu) returns the kernel for a
+// register allocation (CTAs per SM) and a variant (what is recorded, several heads at once, lazy arrivals).
+typedef void (*step_kernel_t)(const Params);
+step_kernel_t step_kernel_of_policy_0(int ctas, int rec, bool bulk, bool lazy);
+step_kernel_t step_kernel_of_policy_1(int ctas, int rec, bool bulk, bool lazy);
+step_kernel_t step_kernel_of_policy_2(int ctas, int rec, bool bulk, bool lazy);
+step_kernel_t step_kernel_of_policy_3(int ctas, int rec, bool bulk, bool lazy);
+step_kernel_t step_kernel_of_policy_4(int ctas, int rec, bool bulk, bool lazy);
+step_kernel_t step_kernel_of_policy_5(int ctas, int rec, bool bulk, bool lazy);
+step_kernel_t step_kernel_of_policy_6(int ctas, int rec, bool bulk, bool lazy);
 
 }  // namespace fcsim_dev
