@@ -30,7 +30,8 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ("paper_2604_11001_b200/csrc/fcsim_device.cuh", "paper_2604_11001_b200/csrc/fcsim.cu")
+SOURCES = ("paper_2604_11001_b200/csrc/fcsim_device.cuh", "paper_2604_11001_b200/csrc/fcsim_step_kernels.cu",
+           "paper_2604_11001_b200/csrc/fcsim.cu")
 CONSTANTS = os.path.join(ROOT, "profiles", "kernel_constants.json")
 METRICS = ("smsp__inst_executed.sum,smsp__issue_active.avg.pct_of_peak_sustained_active,gpu__time_duration.sum,"
            "dram__bytes_read.sum,dram__bytes_write.sum")
