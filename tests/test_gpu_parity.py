@@ -25,7 +25,7 @@ def test_hand_traces_on_gpu(name):
     assert_same(cfg, gpu, orc.run(cfg), cfg.T_max, name)
 
 
-@pytest.mark.parametrize("seed", range(200))
+@pytest.mark.parametrize("seed", range(600))
 def test_random_small_configs(seed):
     cfg = wl.random_small_config(seed, n_replicas=5, T=97)
     gpu = run_gpu(cfg)
@@ -182,7 +182,7 @@ def test_horizon_limit_and_range_errors():
     assert fb.fcsim_query_sizes(late.with_(trace_stride=0, complog_cap=0))["trace"] == 0
 
 
-@pytest.mark.parametrize("seed", range(100))
+@pytest.mark.parametrize("seed", range(250))
 def test_random_medium_configs(seed):
     # preset-sized laws, thousands of slots, every policy: lazy removal, in-place eviction, storage-bound
     # squeezes and resumed launches all occur
