@@ -116,9 +116,9 @@ def test_config2_full():
 
 def test_config3_full():
     cfg = wl.config3()
-    # every 4th group of the 64 x 64 sweep (offset 1: every arrival rate, 16 of the 64 flow-control settings), all
-    # 16 replicas of each: 16 384 replicas over the full horizon
-    groups = range(1, len(cfg.groups), 4)
+    # every 2nd group of the 64 x 64 sweep (offset 1: every arrival rate, 32 of the 64 flow-control settings), all
+    # 16 replicas of each: 32 768 replicas over the full horizon
+    groups = range(1, len(cfg.groups), 2)
     _run_full(cfg, 2000, [16 * g + k for g in groups for k in range(16)], batch=1024)
 
 
